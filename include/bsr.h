@@ -1,0 +1,251 @@
+/*
+ * bsr.h -- C interface of the bounded-state restoration (BSR) library for NVIDIA B200.
+ *
+ * The library restores a complete reusable KV-cache prefix from an external host tier into an
+ * engine's paged KV cache through a staging window of at most W chunks, following the paper's
+ * three-phase protocol (Section 3 "Protocol: Probe, Install, Commit"):
+ *
+ *     bsr_probe      complete candidate hit H(S) as knowledge, not residency
+ *     bsr_restore    bounded installation: |L(t)| <= W live staged chunks (Eq. 3, Eq. 4)
+ *     bsr_commit     expose the advertised prefix only if Q(S) = AND_r AND_g q_{r,g} = 1 (Eq. 6)
+ *     bsr_invalidate whole-prefix invalidation on any failure (Proposition 2)
+ *
+ * Conventions
+ *   - Every function returns an int status: BSR_OK (0) or a negative BSR_ERR_* code.  Nothing
+ *     throws, aborts or exits.  Out-parameters are written only on BSR_OK unless stated.
+ *   - "host" pointers are ordinary CPU addresses; "device" pointers are CUDA device addresses of
+ *     the context's GPU.  The library never frees memory it did not allocate.
+ *   - Handles (bsr_ctx, bsr_req) are opaque.  A context is bound to one GPU.  Calls on one context
+ *     may come from any thread; restores on one context are serialised by a context-wide lock
+ *     (Section 3 "Install locally": concurrent requests must not multiply the staging budget).
+ *   - All integer arithmetic of the method is unsigned, modulo 2^64.
+ *
+ * Functions the paper leaves open and this library defines (documented at each call): the chunk
+ * digest and prefix-key chain, the per-(rank, chunk, group) checksum, the chunk byte layout, the
+ * paged layout and the validity-bitmap layout.
+ */
+#ifndef BSR_H_
+#define BSR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define BSR_CHUNK_TOKENS 256u /* Section 4 "System topology": the chunk is 256 tokens        */
+#define BSR_MAX_GROUPS 8u     /* allocator groups per registration                             */
+#define BSR_MAX_RANKS 8u      /* TP rank slices per context                                    */
+
+enum {
+  BSR_OK = 0,
+  BSR_ERR_INVALID = -1,  /* bad argument, W = 0, unknown handle                                */
+  BSR_ERR_MISSING = -2,  /* a chunk of the advertised prefix is not in the tier                */
+  BSR_ERR_CHECKSUM = -3, /* a staged group segment does not match its stored checksum          */
+  BSR_ERR_TIMEOUT = -4,  /* a fill, copy or install did not finish within timeout_ms           */
+  BSR_ERR_TRANSFER = -5, /* the tier read or the host-to-device copy reported an error         */
+  BSR_ERR_NOMEM = -6,    /* a host or device allocation failed                                 */
+  BSR_ERR_ALIGN = -7,    /* bytes_per_token not a multiple of 16, or a pointer not 16-B aligned */
+  BSR_ERR_STATE = -8,    /* call not legal in this state (e.g. register after first restore)   */
+  BSR_ERR_CUDA = -9      /* a CUDA runtime call failed; see bsr_last_error                     */
+};
+
+typedef struct bsr_ctx bsr_ctx;
+typedef struct bsr_req bsr_req;
+
+/* Where a tier object's bytes live. */
+enum {
+  BSR_LOC_HOST = 0,  /* pageable or pinned host memory: restored through the pinned ring       */
+  BSR_LOC_DEVICE = 1 /* already in this GPU's memory: installed in place, no staging is used   */
+};
+
+/* Which install kernel bsr_restore launches. */
+enum { BSR_INSTALL_AUTO = 0, BSR_INSTALL_VECTOR = 1, BSR_INSTALL_BULK = 2 };
+
+typedef struct bsr_config {
+  uint32_t window_chunks;     /* W >= 1: pinned staging slots per rank (Eq. 3).  W = 0, the paper's
+                                 legacy whole-plan mode (Table 1), is rejected                  */
+  uint32_t n_ranks;           /* R: TP rank slices restored by this context, 1..BSR_MAX_RANKS   */
+  uint32_t chunk_tokens;      /* must be BSR_CHUNK_TOKENS                                        */
+  uint32_t load_concurrency;  /* threads copying tier objects into staging slots (Table 1 "FS
+                                 load concurrency": changes throughput, never W or the peak)     */
+  uint32_t dev_staging_depth; /* D >= 1 device staging buffers per rank (bounded auxiliary state,
+                                 M_aux of Eq. 4; independent of the prefix length)               */
+  uint32_t timeout_ms;        /* deadline of one bsr_restore call; 0 = 30,000                    */
+  uint32_t slot_align;        /* staging slot size = chunk bytes rounded up to this; 0 = 4096    */
+  int32_t device;             /* CUDA device ordinal                                             */
+  uint64_t reg_id;            /* registration identity mixed into every prefix key               */
+  uint32_t install_variant;   /* BSR_INSTALL_*                                                   */
+  uint32_t time_kernels;      /* nonzero: bracket every install launch with CUDA events and
+                                 accumulate bsr_stats.install_kernel_ms                          */
+} bsr_config;
+
+typedef struct bsr_group_desc {
+  uint32_t block_tokens;    /* tokens per paged block; must divide 256                           */
+  uint32_t num_phys_blocks; /* size of the group's physical block pool                           */
+} bsr_group_desc;
+
+typedef struct bsr_tensor_desc {
+  uint32_t group;           /* allocator group of this tensor                                    */
+  uint32_t bytes_per_token; /* multiple of 16                                                    */
+  void *dev_base;           /* device, caller-owned, 16-byte aligned, at least
+                               num_phys_blocks * block_tokens * bytes_per_token bytes            */
+} bsr_tensor_desc;
+
+typedef struct bsr_stats {
+  uint64_t peak_staging_bytes[BSR_MAX_RANKS];   /* max over time of live slots x slot bytes (Eq. 1) */
+  uint64_t ring_bytes_allocated[BSR_MAX_RANKS]; /* pinned ring size: W x slot bytes                  */
+  uint64_t bytes_filled[BSR_MAX_RANKS];         /* tier -> slot                                      */
+  uint64_t bytes_h2d[BSR_MAX_RANKS];            /* slot -> device staging                            */
+  uint64_t bytes_installed[BSR_MAX_RANKS];      /* verified and scattered                            */
+  uint64_t slot_bytes;                          /* staging footprint of one chunk                    */
+  uint64_t dev_aux_bytes;                       /* device staging + kernel scratch, all ranks        */
+  uint64_t windows;                             /* passes over the ring: K = ceil(N / W)             */
+  uint64_t tier_bytes_read_by_probe;            /* stays 0: probe touches the index only             */
+  uint64_t kernel_launches;                     /* kernels of this library launched                  */
+  uint64_t h2d_copies;                          /* cudaMemcpyAsync calls issued                      */
+  uint64_t install_launches;                    /* install kernel launches                           */
+  double install_kernel_ms;                     /* sum of their device durations (time_kernels)      */
+  double last_restore_ms;                       /* host wall time of the last bsr_restore            */
+} bsr_stats;
+
+/* ---- context ------------------------------------------------------------------------------- */
+
+/* Creates a context on cfg->device.  Allocates nothing proportional to a prefix; the pinned ring
+ * (W slots per rank) and the device staging buffers are allocated at the first restore, when the
+ * chunk size is known.  Errors: INVALID (W = 0, ranks out of range, chunk_tokens != 256), CUDA. */
+int bsr_ctx_create(const bsr_config *cfg, bsr_ctx **out);
+
+/* Destroys the context, its ring, staging, index and any request still alive. */
+int bsr_ctx_destroy(bsr_ctx *ctx);
+
+/* Text of the last CUDA or argument error seen by this context (never NULL; valid until the next
+ * failing call on the context). */
+const char *bsr_last_error(bsr_ctx *ctx);
+
+/* ---- registration (Section 4: registered tensors in allocator groups, per TP rank) -------- */
+
+/* Registers rank's paged pools.  groups[G] and tensors[L] are host arrays, copied.  Tensors must
+ * be listed group-major (all of group 0, then group 1, ...).  All ranks must register the same
+ * geometry; only dev_base differs.
+ *
+ * Chunk byte layout (defined here, the paper only says a chunk "spans the registered per-rank state
+ * of its token range"): groups in order; inside a group its tensors in registration order; per
+ * tensor 256 tokens x bytes_per_token, token-major.
+ * Paged layout: tensor l is an array [num_phys_blocks][block_tokens][bytes_per_token]; logical block
+ * j of the request maps to physical block table[j] of the tensor's group.
+ * Errors: INVALID, ALIGN, STATE (after the first restore). */
+int bsr_register(bsr_ctx *ctx, uint32_t rank, const bsr_group_desc *groups, uint32_t n_groups,
+                 const bsr_tensor_desc *tensors, uint32_t n_tensors);
+
+/* Bytes of one chunk and of one staging slot under the current registration. */
+int bsr_chunk_bytes(bsr_ctx *ctx, uint64_t *chunk_bytes, uint64_t *slot_bytes);
+
+/* ---- external tier + chunk index ---------------------------------------------------------- */
+
+/* Adds (or replaces) the object `key` of `rank`.  `data` (host or device per `location`) is
+ * BORROWED: the caller keeps it alive and unmodified for as long as the key is present (tests
+ * corrupt it on purpose).  len must equal the chunk bytes.  group_ck[G] (host) are the checksums
+ * of the G group segments; NULL makes the library compute them now on the GPU (store path).
+ *
+ * Checksum (defined here; Table 1 says "verify" without a formula): over the little-endian 32-bit
+ * words w_k of a group's segment, k from the segment start, CK = sum_k w_k * (2k + 1) mod 2^64.
+ * Errors: INVALID, STATE (no registration), CUDA. */
+int bsr_tier_put(bsr_ctx *ctx, uint32_t rank, uint64_t key, const void *data, size_t len,
+                 const uint64_t *group_ck, int location);
+
+/* Removes a key (no error if absent).  A chunk may vanish between probe and restore; the restore
+ * then fails closed with BSR_ERR_MISSING. */
+int bsr_tier_remove(bsr_ctx *ctx, uint32_t rank, uint64_t key);
+
+/* Reads back the stored checksums of a key into out[G] (host).  MISSING if absent. */
+int bsr_tier_checksums(bsr_ctx *ctx, uint32_t rank, uint64_t key, uint64_t *out);
+
+/* ---- probe (Section 3 "Probe globally") ---------------------------------------------------- */
+
+/* Computes, on the GPU, one digest per full 256-token chunk and chains them into prefix keys, then
+ * looks every key up in the chunk index of every rank.
+ *
+ *   mix64(x): x += PHI; x = (x ^ x>>32) * PHI; x = (x ^ x>>29) * PHI; return x ^ x>>32
+ *             with PHI = 0x9E3779B97F4A7C15
+ *   d_i  = sum_{j<256} mix64( ((u64)(u32)tok[256 i + j] << 32 | j) ^ salt )
+ *   k_-1 = mix64(salt ^ mix64(reg_id)),   k_i = mix64(k_{i-1} ^ d_i)
+ *
+ * tok: n_tok int32 ids, host or device per tok_on_device; the trailing n_tok % 256 are ignored.
+ * keys_out[N] (host, may be NULL), hit_bitmap_out[ceil(N/64)] (host, may be NULL; bit i = every
+ * rank holds key i), n_hit_chunks = length of the longest all-hit prefix.  N = n_tok / 256.
+ * Probe reads no payload byte, takes no staging slot and keeps no lock or reference after return.
+ * Errors: INVALID, STATE, CUDA. */
+int bsr_probe(bsr_ctx *ctx, const int32_t *tok, size_t n_tok, int tok_on_device, uint64_t salt,
+              uint64_t *keys_out, uint64_t *hit_bitmap_out, uint32_t *n_hit_chunks);
+
+/* ---- request: advertised prefix and destination blocks (Fig. 2, second box) -------------- */
+
+/* The caller plays the scheduler: it advertises the first n_adv_chunks keys and has allocated the
+ * destination blocks.  block_tables is a host array of R*G host pointers, entry r*G+g pointing at
+ * n_adv_chunks * 256 / block_tokens[g] int32 physical block ids.  Tables are validated (ids in
+ * range, no duplicates within a table) and copied to the device.  Errors: INVALID, NOMEM, CUDA. */
+int bsr_req_create(bsr_ctx *ctx, const uint64_t *keys, uint32_t n_adv_chunks,
+                   const int32_t *const *block_tables, bsr_req **out);
+
+int bsr_req_release(bsr_ctx *ctx, bsr_req *req);
+
+/* ---- restore (Section 2 "Bounded installation", Section 3 "Install locally") -------------- */
+
+/* Installs the advertised prefix of every rank.  Chunk i of rank r is copied from the tier into
+ * pinned slot i mod W of r's ring (at most W slots live per rank, a slot is live from before its
+ * fill until its install has been observed complete), copied to a device staging buffer on the
+ * library's copy stream, then verified and scattered through the block tables by the install
+ * kernel on `cuda_stream` (a cudaStream_t, or NULL for a stream owned by the library).  The first
+ * missing key, checksum mismatch, transfer error or deadline overrun stops admission, drains what
+ * is in flight, invalidates the whole request and is returned.  Blocking; on return no slot is
+ * live and every kernel of the call has finished.
+ * Returns BSR_OK iff every (rank, group, chunk) was verified and installed. */
+int bsr_restore(bsr_ctx *ctx, bsr_req *req, void *cuda_stream);
+
+/* ---- commit / invalidate (Section 3 "Commit at request semantics", Eq. 6, Proposition 2) -- */
+
+/* exposed_chunks = n_adv_chunks iff a restore of the request completed and all validity bits are
+ * set; otherwise the request is invalidated and 0 is exposed (a zero-reuse outcome is an answer,
+ * not an API error).  Idempotent. */
+int bsr_commit(bsr_ctx *ctx, bsr_req *req, uint32_t *exposed_chunks);
+
+#define BSR_SCRUB 1u /* also zero-fill every destination block of the request, all groups/ranks */
+
+/* Clears the whole validity bitmap (healthy ranks and groups included); afterwards commit yields
+ * 0.  Idempotent. */
+int bsr_invalidate(bsr_ctx *ctx, bsr_req *req, unsigned flags);
+
+/* ---- observability ------------------------------------------------------------------------ */
+
+/* Validity bitmap: bit (r, g, i) lives in word (r*G + g) * ceil(n_adv/64) + i/64 at position
+ * i % 64.  `words` must be at least R*G*ceil(n_adv/64). */
+int bsr_req_bitmap(bsr_ctx *ctx, bsr_req *req, uint64_t *out, size_t words);
+
+/* Checksums the install kernel computed, out[(r*G + g) * n_adv + i]; 0 where not installed. */
+int bsr_req_checksums(bsr_ctx *ctx, bsr_req *req, uint64_t *out, size_t count);
+
+int bsr_get_stats(bsr_ctx *ctx, bsr_stats *out);
+int bsr_reset_stats(bsr_ctx *ctx);
+
+/* ---- host-side failure injection (tests) -------------------------------------------------- */
+
+enum {
+  BSR_INJECT_NONE = 0,
+  BSR_INJECT_CORRUPT_SLOT = 1, /* flip one word of (rank, group, chunk) in the pinned slot after
+                                  the fill, before the device copy                             */
+  BSR_INJECT_FILL_ERROR = 2,   /* the tier read of (rank, chunk) reports a transfer error      */
+  BSR_INJECT_FILL_STALL = 3    /* the tier read of (rank, chunk) does not finish before the
+                                  deadline                                                     */
+};
+
+/* Arms one fault for the next restore (one shot; BSR_INJECT_NONE disarms).  Acts on host memory
+ * and host threads only; the GPU is never made to fault, trap or spin. */
+int bsr_test_inject(bsr_ctx *ctx, int kind, uint32_t rank, uint32_t group, uint32_t chunk,
+                    uint64_t seed);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BSR_H_ */
