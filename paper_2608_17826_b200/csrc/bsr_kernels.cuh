@@ -1,0 +1,279 @@
+// Device code of the BSR library (sm_100a): probe, install (verify + scatter), scrub.
+//
+// Pure data movement and 64-bit integer sums: no tensor cores.  Every byte has one reader, so no
+// cluster multicast is used anywhere; bulk copies are plain per-CTA 1-D copies.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#define BSR_K_MAX_GROUPS 8
+#define BSR_K_MAX_BATCH 64        // chunk descriptors per install launch
+#define BSR_K_TILE_MAX 16384u     // largest tile in bytes (one bulk-copy stage)
+#define BSR_K_PHI 0x9E3779B97F4A7C15ull
+
+// ---------------------------------------------------------------------------------------------
+// shared structs (host fills, device reads)
+// ---------------------------------------------------------------------------------------------
+
+// One piece of one destination run.  A chunk's tile table is the same for every chunk and rank of
+// a registration: only the source base, the block-table row and the tensor base pointers change.
+struct __align__(16) BsrTile {
+  uint32_t src_off;    // byte offset inside the chunk (multiple of 16)
+  uint32_t bytes;      // tile length (multiple of 16, <= BSR_K_TILE_MAX)
+  uint32_t dst_off;    // byte offset inside the destination block run
+  uint32_t word0;      // index of the tile's first 32-bit word inside its group segment
+  uint32_t run_bytes;  // block_tokens * bytes_per_token of the tensor
+  uint16_t tensor;     // registration index l
+  uint8_t group;       // allocator group g
+  uint8_t blk;         // logical block of the chunk, 0 .. 256/block_tokens - 1
+  uint32_t pad[2];
+};
+static_assert(sizeof(BsrTile) == 32, "tile is two 16-byte loads");
+
+struct BsrChunkDesc {
+  const uint8_t *src;  // device address of the staged chunk
+  uint32_t chunk;      // index i in the advertised prefix
+  uint32_t rank;       // TP rank slice r
+  uint64_t expect[BSR_K_MAX_GROUPS];  // stored checksums of the group segments
+};
+
+struct BsrInstallParams {
+  const BsrTile *tiles;
+  uint32_t n_tiles;    // tiles per chunk
+  uint32_t n_chunks;   // descriptors in this launch
+  uint32_t n_groups;
+  uint32_t n_tensors;
+  uint32_t n_adv;      // advertised chunks of the request (row length of ck_out / verdict)
+  uint32_t scatter;    // 0: checksum only (store path), 1: verify + scatter
+  const uint64_t *tensor_base;   // [R][L] device addresses of the paged tensors
+  const int32_t *const *tables;  // [R*G] device pointers to the request's block tables
+  uint32_t blocks_per_chunk[BSR_K_MAX_GROUPS];
+  uint64_t *acc;             // scratch [BSR_K_MAX_BATCH][BSR_K_MAX_GROUPS]; zero on entry, zeroed on exit
+  unsigned int *ctas_done;   // scratch counter; zero on entry, zeroed on exit
+  unsigned int *err_flag;    // set to nonzero if a bounded wait gave up (bulk variant)
+  uint64_t *ck_out;          // [(r*G + g) * n_adv + i] computed checksum
+  uint32_t *verdict;         // same index: 1 verified, 2 mismatch
+  BsrChunkDesc chunk[BSR_K_MAX_BATCH];
+};
+
+// ---------------------------------------------------------------------------------------------
+// helpers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint64_t bsr_mix64(uint64_t x) {
+  x += BSR_K_PHI;
+  x = (x ^ (x >> 32)) * BSR_K_PHI;
+  x = (x ^ (x >> 29)) * BSR_K_PHI;
+  return x ^ (x >> 32);
+}
+
+__device__ __forceinline__ uint64_t bsr_warp_sum(uint64_t v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Contribution of one 16-byte vector whose first word has index k inside the segment:
+// sum_{q<4} w_q * (2(k+q) + 1), each product 32x32 -> 64 bits.
+__device__ __forceinline__ uint64_t bsr_ck_vec(uint4 w, uint32_t k) {
+  const uint32_t wt = 2u * k + 1u;
+  uint64_t s = (uint64_t)w.x * (uint64_t)wt;
+  s += (uint64_t)w.y * (uint64_t)(wt + 2u);
+  s += (uint64_t)w.z * (uint64_t)(wt + 4u);
+  s += (uint64_t)w.w * (uint64_t)(wt + 6u);
+  return s;
+}
+
+__device__ __forceinline__ uint4 bsr_ld_stream(const uint4 *p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+__device__ __forceinline__ void bsr_st_stream(uint4 *p, uint4 v) {
+  asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z),
+               "r"(v.w)
+               : "memory");
+}
+
+// Block-wide sum of per-thread partials, added once into *dst (sums mod 2^64 commute, so the
+// order of the atomics cannot change the result).
+template <int THREADS>
+__device__ __forceinline__ void bsr_block_flush(uint64_t v, uint64_t *dst, uint64_t *smem) {
+  v = bsr_warp_sum(v);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (lane == 0) smem[warp] = v;
+  __syncthreads();
+  if (warp == 0) {
+    uint64_t t = (lane < THREADS / 32) ? smem[lane] : 0ull;
+    t = bsr_warp_sum(t);
+    if (lane == 0) atomicAdd((unsigned long long *)dst, (unsigned long long)t);
+  }
+  __syncthreads();
+}
+
+// The last CTA to finish compares every (chunk, group) sum of the launch with the stored checksum,
+// publishes sum and verdict, and leaves the scratch zeroed for the next launch.
+template <int THREADS>
+__device__ __forceinline__ void bsr_install_finish(const BsrInstallParams &p) {
+  __shared__ int is_last;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const unsigned prev = atomicAdd(p.ctas_done, 1u);
+    is_last = (prev == gridDim.x - 1u);
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  const uint32_t G = p.n_groups;
+  for (uint32_t idx = threadIdx.x; idx < p.n_chunks * G; idx += THREADS) {
+    const uint32_t c = idx / G, g = idx - c * G;
+    uint64_t *a = p.acc + c * BSR_K_MAX_GROUPS + g;
+    const uint64_t s = __ldcg((const unsigned long long *)a);
+    *a = 0ull;
+    const BsrChunkDesc &cd = p.chunk[c];
+    const size_t o = ((size_t)cd.rank * G + g) * p.n_adv + cd.chunk;
+    p.ck_out[o] = s;
+    p.verdict[o] = (s == cd.expect[g]) ? 1u : 2u;
+  }
+  if (threadIdx.x == 0) *p.ctas_done = 0u;
+}
+
+// ---------------------------------------------------------------------------------------------
+// install, vector variant: 16-byte streaming loads and stores, UNROLL vectors in flight per thread
+// ---------------------------------------------------------------------------------------------
+template <int THREADS, int UNROLL>
+__global__ void __launch_bounds__(THREADS)
+bsr_install_vec_kernel(const __grid_constant__ BsrInstallParams p) {
+  __shared__ uint64_t red[THREADS / 32];
+  const uint32_t total = p.n_chunks * p.n_tiles;
+  uint64_t sum = 0;
+  int cur_c = -1, cur_g = -1;
+  for (uint32_t w = blockIdx.x; w < total; w += gridDim.x) {
+    const uint32_t c = w / p.n_tiles, t = w - c * p.n_tiles;
+    const uint4 *tp = reinterpret_cast<const uint4 *>(p.tiles + t);
+    const uint4 t0 = __ldg(tp), t1 = __ldg(tp + 1);
+    const uint32_t src_off = t0.x, bytes = t0.y, dst_off = t0.z, word0 = t0.w;
+    const uint32_t run_bytes = t1.x, tensor = t1.y & 0xffffu, g = (t1.y >> 16) & 0xffu,
+                   blk = t1.y >> 24;
+    if ((int)c != cur_c || (int)g != cur_g) {  // block-uniform
+      if (cur_c >= 0) bsr_block_flush<THREADS>(sum, p.acc + cur_c * BSR_K_MAX_GROUPS + cur_g, red);
+      sum = 0;
+      cur_c = (int)c;
+      cur_g = (int)g;
+    }
+    const BsrChunkDesc &cd = p.chunk[c];
+    const uint4 *src = reinterpret_cast<const uint4 *>(cd.src + src_off);
+    uint4 *dst = nullptr;
+    if (p.scatter) {
+      const int32_t *table = p.tables[cd.rank * p.n_groups + g];
+      const int32_t phys = __ldg(table + (size_t)cd.chunk * p.blocks_per_chunk[g] + blk);
+      const uint64_t base = __ldg(p.tensor_base + (size_t)cd.rank * p.n_tensors + tensor);
+      dst = reinterpret_cast<uint4 *>(base + (uint64_t)phys * run_bytes + dst_off);
+    }
+    const uint32_t nvec = bytes >> 4;
+    for (uint32_t v0 = threadIdx.x; v0 < nvec; v0 += THREADS * UNROLL) {
+      uint4 r[UNROLL];
+#pragma unroll
+      for (int u = 0; u < UNROLL; ++u) {
+        const uint32_t v = v0 + u * THREADS;
+        if (v < nvec) r[u] = bsr_ld_stream(src + v);
+      }
+#pragma unroll
+      for (int u = 0; u < UNROLL; ++u) {
+        const uint32_t v = v0 + u * THREADS;
+        if (v < nvec) {
+          if (dst) bsr_st_stream(dst + v, r[u]);
+          sum += bsr_ck_vec(r[u], word0 + 4u * v);
+        }
+      }
+    }
+  }
+  if (cur_c >= 0) bsr_block_flush<THREADS>(sum, p.acc + cur_c * BSR_K_MAX_GROUPS + cur_g, red);
+  bsr_install_finish<THREADS>(p);
+}
+
+// ---------------------------------------------------------------------------------------------
+// probe: chunk digests (one warp per chunk), then the last block chains the prefix keys
+// ---------------------------------------------------------------------------------------------
+#define BSR_K_PROBE_THREADS 256
+#define BSR_K_CHAIN_TILE 2048
+
+__global__ void __launch_bounds__(BSR_K_PROBE_THREADS)
+bsr_probe_kernel(const int32_t *__restrict__ tok, uint32_t n_chunks, uint64_t salt, uint64_t k_init,
+                 uint64_t *digests /* scratch [n_chunks] */, unsigned int *blocks_done /* scratch */,
+                 uint64_t *keys /* out [n_chunks] */) {
+  __shared__ uint64_t tile[BSR_K_CHAIN_TILE];
+  __shared__ int is_last;
+  const uint32_t lane = threadIdx.x & 31u;
+  const uint32_t chunk = blockIdx.x * (BSR_K_PROBE_THREADS / 32) + (threadIdx.x >> 5);
+  if (chunk < n_chunks) {
+    const int4 *base = reinterpret_cast<const int4 *>(tok + (size_t)chunk * 256u);
+    uint64_t s = 0;
+#pragma unroll
+    for (uint32_t m = 0; m < 2; ++m) {
+      const uint32_t q = m * 32u + lane;  // int4 index inside the chunk: tokens 4q .. 4q+3
+      const int4 t = __ldg(base + q);
+      const uint32_t j = 4u * q;
+      s += bsr_mix64((((uint64_t)(uint32_t)t.x << 32) | (uint64_t)(j + 0u)) ^ salt);
+      s += bsr_mix64((((uint64_t)(uint32_t)t.y << 32) | (uint64_t)(j + 1u)) ^ salt);
+      s += bsr_mix64((((uint64_t)(uint32_t)t.z << 32) | (uint64_t)(j + 2u)) ^ salt);
+      s += bsr_mix64((((uint64_t)(uint32_t)t.w << 32) | (uint64_t)(j + 3u)) ^ salt);
+    }
+    s = bsr_warp_sum(s);
+    if (lane == 0) digests[chunk] = s;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    is_last = (atomicAdd(blocks_done, 1u) == gridDim.x - 1u);
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  // serial chain k_i = mix64(k_{i-1} ^ d_i), digests staged through shared memory
+  uint64_t k = k_init;
+  for (uint32_t base_i = 0; base_i < n_chunks; base_i += BSR_K_CHAIN_TILE) {
+    const uint32_t n = min((uint32_t)BSR_K_CHAIN_TILE, n_chunks - base_i);
+    for (uint32_t i = threadIdx.x; i < n; i += BSR_K_PROBE_THREADS)
+      tile[i] = __ldcg((const unsigned long long *)(digests + base_i + i));
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      for (uint32_t i = 0; i < n; ++i) {
+        k = bsr_mix64(k ^ tile[i]);
+        keys[base_i + i] = k;
+      }
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *blocks_done = 0u;
+}
+
+// ---------------------------------------------------------------------------------------------
+// scrub: zero-fill every destination block run of a request (all ranks, groups, tensors)
+// grid.y = r * L + l, grid.x strides over the logical blocks of the tensor's group
+// ---------------------------------------------------------------------------------------------
+struct BsrScrubParams {
+  const uint64_t *tensor_base;   // [R][L]
+  const int32_t *const *tables;  // [R*G]
+  const uint32_t *tensor_group;  // [L]
+  const uint32_t *tensor_run;    // [L] run bytes
+  uint32_t n_tensors, n_groups, n_adv;
+  uint32_t blocks_per_chunk[BSR_K_MAX_GROUPS];
+};
+
+__global__ void __launch_bounds__(256) bsr_scrub_kernel(const __grid_constant__ BsrScrubParams p) {
+  const uint32_t r = blockIdx.y / p.n_tensors, l = blockIdx.y - r * p.n_tensors;
+  const uint32_t g = p.tensor_group[l], run = p.tensor_run[l];
+  const uint32_t n_logical = p.n_adv * p.blocks_per_chunk[g];
+  const int32_t *table = p.tables[r * p.n_groups + g];
+  const uint64_t base = p.tensor_base[(size_t)r * p.n_tensors + l];
+  const uint4 z = make_uint4(0, 0, 0, 0);
+  for (uint32_t j = blockIdx.x; j < n_logical; j += gridDim.x) {
+    uint4 *dst = reinterpret_cast<uint4 *>(base + (uint64_t)__ldg(table + j) * run);
+    for (uint32_t v = threadIdx.x; v < (run >> 4); v += 256) dst[v] = z;
+  }
+}

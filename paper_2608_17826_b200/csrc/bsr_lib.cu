@@ -1,0 +1,1108 @@
+// Host side of the BSR library: context, registration, chunk index, probe, the W-slot window
+// pipeline (pinned ring -> copy stream -> device staging -> install kernel), commit, invalidate.
+// The C interface is declared in include/bsr.h.
+#include "../../include/bsr.h"
+
+#include <atomic>
+#include <chrono>
+#include <condition_variable>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <string>
+#include <thread>
+#include <unordered_map>
+#include <vector>
+
+#include "bsr_kernels.cuh"
+
+namespace {
+
+using Clock = std::chrono::steady_clock;
+
+constexpr int kInstallThreads = 256;
+constexpr int kInstallUnroll = 4;
+constexpr int kLaunchSlots = 8;  // independent scratch sets for install launches in flight
+constexpr uint32_t kSmCount = 148;
+
+struct TierObj {
+  const uint8_t *data;
+  size_t len;
+  int loc;
+  uint64_t ck[BSR_MAX_GROUPS];
+};
+
+struct TensorReg {
+  uint32_t group;
+  uint32_t bytes_per_token;
+  uint64_t base[BSR_MAX_RANKS];
+};
+
+struct Inject {
+  int kind = BSR_INJECT_NONE;
+  uint32_t rank = 0, group = 0, chunk = 0;
+  uint64_t seed = 0;
+};
+
+}  // namespace
+
+struct bsr_req {
+  bsr_ctx *ctx = nullptr;
+  uint32_t n_adv = 0;
+  std::vector<uint64_t> keys;
+  std::vector<std::vector<int32_t>> tables;  // [R*G]
+  int32_t *d_tables = nullptr;               // all tables, flat
+  const int32_t **d_table_ptrs = nullptr;    // [R*G] device pointers into d_tables
+  uint64_t *h_ck = nullptr;                  // pinned, device-visible: [(R*G)][n_adv]
+  uint32_t *h_verdict = nullptr;             // pinned, device-visible
+  uint64_t *d_ck = nullptr;                  // device aliases of the two arrays above
+  uint32_t *d_verdict = nullptr;
+  std::vector<uint64_t> bitmap;              // [R*G][words]
+  uint32_t words = 0;
+  bool restored = false;
+  bool failed = false;
+};
+
+struct bsr_ctx {
+  bsr_config cfg{};
+  std::mutex mu;          // registration, tier index, stats, error text
+  std::mutex restore_mu;  // one bounded restore at a time
+  std::string err;
+
+  // registration
+  uint32_t G = 0, L = 0;
+  bool rank_registered[BSR_MAX_RANKS] = {};
+  std::vector<bsr_group_desc> groups;
+  std::vector<TensorReg> tensors;
+  uint64_t chunk_bytes = 0, slot_bytes = 0;
+  uint64_t seg_begin[BSR_MAX_GROUPS] = {}, seg_bytes[BSR_MAX_GROUPS] = {};
+  bool finalized = false;
+  std::vector<BsrTile> h_tiles;
+  BsrTile *d_tiles = nullptr;
+  uint64_t *d_tensor_base = nullptr;
+  uint32_t *d_tensor_group = nullptr, *d_tensor_run = nullptr;
+
+  // tier + index
+  std::unordered_map<uint64_t, TierObj> tier[BSR_MAX_RANKS];
+  uint8_t *d_put_stage = nullptr;
+  uint64_t *h_put_ck = nullptr, *d_put_ck = nullptr;  // pinned [G] sums + verdict dump
+  uint32_t *h_put_verdict = nullptr, *d_put_verdict = nullptr;
+
+  // streams and scratch
+  cudaStream_t copy_stream = nullptr, own_stream = nullptr;
+  uint64_t *d_acc = nullptr;        // [kLaunchSlots][BATCH][GROUPS]
+  unsigned int *d_counters = nullptr;  // [kLaunchSlots] install + [1] probe + [1] err flag
+  uint64_t launch_seq = 0;
+
+  // probe scratch (grown on demand)
+  int32_t *d_tok = nullptr;
+  uint64_t *d_digests = nullptr, *d_keys = nullptr, *h_keys = nullptr;
+  size_t probe_cap_chunks = 0;
+
+  // ring
+  bool ring_ready = false;
+  uint8_t *ring[BSR_MAX_RANKS] = {};
+  uint8_t *dstage[BSR_MAX_RANKS] = {};
+  std::vector<cudaEvent_t> ev_h2d, ev_inst, ev_start;  // [R*D]
+  std::vector<cudaEvent_t> ev_batch_start, ev_batch_stop;  // resident mode
+
+  // filler pool
+  std::vector<std::thread> fillers;
+  std::mutex fill_mu;
+  std::condition_variable fill_cv;
+  bool fill_shutdown = false;
+  // state of the restore in progress, guarded by fill_mu unless atomic
+  bsr_req *cur_req = nullptr;
+  uint32_t fill_total = 0, fill_admitted = 0, fill_next = 0;
+  std::atomic<bool> fill_abort{false};
+  Clock::time_point fill_deadline;
+  std::vector<std::atomic<int>> *task_state = nullptr;  // 0 pending, 1 ready, <0 error
+  std::vector<TierObj> *task_obj = nullptr;
+  uint32_t fill_active = 0;
+
+  Inject inject;
+  bsr_stats st{};
+  uint64_t live[BSR_MAX_RANKS] = {};
+};
+
+namespace {
+
+int fail(bsr_ctx *c, int code, const char *fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  if (c) {
+    std::lock_guard<std::mutex> g(c->mu);
+    c->err = buf;
+  }
+  return code;
+}
+
+#define CU(c, call)                                                                     \
+  do {                                                                                  \
+    cudaError_t e_ = (call);                                                            \
+    if (e_ != cudaSuccess)                                                              \
+      return fail((c), BSR_ERR_CUDA, "%s: %s (%s:%d)", #call, cudaGetErrorString(e_),   \
+                  __FILE__, __LINE__);                                                  \
+  } while (0)
+
+uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+
+// ---- registration -> tile table ----------------------------------------------------------------
+int finalize_registration(bsr_ctx *c) {
+  if (c->finalized) return BSR_OK;
+  if (c->L == 0) return fail(c, BSR_ERR_STATE, "no registration");
+  for (uint32_t r = 0; r < c->cfg.n_ranks; ++r)
+    if (!c->rank_registered[r]) return fail(c, BSR_ERR_STATE, "rank %u is not registered", r);
+  CU(c, cudaSetDevice(c->cfg.device));
+  std::vector<uint32_t> tgroup(c->L), trun(c->L);
+  uint64_t off = 0;
+  c->h_tiles.clear();
+  for (uint32_t l = 0; l < c->L; ++l) {
+    const TensorReg &t = c->tensors[l];
+    const uint32_t B = c->groups[t.group].block_tokens;
+    const uint32_t nb = BSR_CHUNK_TOKENS / B;
+    const uint64_t run = (uint64_t)B * t.bytes_per_token;
+    tgroup[l] = t.group;
+    trun[l] = (uint32_t)run;
+    const uint32_t nsplit = (uint32_t)((run + BSR_K_TILE_MAX - 1) / BSR_K_TILE_MAX);
+    const uint32_t piece = (uint32_t)round_up((run + nsplit - 1) / nsplit, 128);
+    for (uint32_t b = 0; b < nb; ++b) {
+      for (uint64_t s = 0; s < run; s += piece) {
+        BsrTile tl{};
+        tl.src_off = (uint32_t)(off + b * run + s);
+        tl.bytes = (uint32_t)((run - s < piece) ? run - s : piece);
+        tl.dst_off = (uint32_t)s;
+        tl.word0 = (uint32_t)((tl.src_off - c->seg_begin[t.group]) / 4);
+        tl.run_bytes = (uint32_t)run;
+        tl.tensor = (uint16_t)l;
+        tl.group = (uint8_t)t.group;
+        tl.blk = (uint8_t)b;
+        c->h_tiles.push_back(tl);
+      }
+    }
+    off += (uint64_t)BSR_CHUNK_TOKENS * t.bytes_per_token;
+  }
+  std::vector<uint64_t> bases((size_t)c->cfg.n_ranks * c->L);
+  for (uint32_t r = 0; r < c->cfg.n_ranks; ++r)
+    for (uint32_t l = 0; l < c->L; ++l) bases[(size_t)r * c->L + l] = c->tensors[l].base[r];
+  CU(c, cudaMalloc(&c->d_tiles, c->h_tiles.size() * sizeof(BsrTile)));
+  CU(c, cudaMemcpy(c->d_tiles, c->h_tiles.data(), c->h_tiles.size() * sizeof(BsrTile),
+                   cudaMemcpyHostToDevice));
+  CU(c, cudaMalloc(&c->d_tensor_base, bases.size() * 8));
+  CU(c, cudaMemcpy(c->d_tensor_base, bases.data(), bases.size() * 8, cudaMemcpyHostToDevice));
+  CU(c, cudaMalloc(&c->d_tensor_group, c->L * 4));
+  CU(c, cudaMemcpy(c->d_tensor_group, tgroup.data(), c->L * 4, cudaMemcpyHostToDevice));
+  CU(c, cudaMalloc(&c->d_tensor_run, c->L * 4));
+  CU(c, cudaMemcpy(c->d_tensor_run, trun.data(), c->L * 4, cudaMemcpyHostToDevice));
+  c->st.dev_aux_bytes += c->h_tiles.size() * sizeof(BsrTile) + bases.size() * 8 + c->L * 8;
+  c->finalized = true;
+  return BSR_OK;
+}
+
+void fill_params(bsr_ctx *c, BsrInstallParams &p, uint32_t slot) {
+  p.tiles = c->d_tiles;
+  p.n_tiles = (uint32_t)c->h_tiles.size();
+  p.n_groups = c->G;
+  p.n_tensors = c->L;
+  p.tensor_base = c->d_tensor_base;
+  for (uint32_t g = 0; g < c->G; ++g)
+    p.blocks_per_chunk[g] = BSR_CHUNK_TOKENS / c->groups[g].block_tokens;
+  p.acc = c->d_acc + (size_t)slot * BSR_K_MAX_BATCH * BSR_K_MAX_GROUPS;
+  p.ctas_done = c->d_counters + slot;
+  p.err_flag = c->d_counters + kLaunchSlots + 1;
+}
+
+uint32_t install_grid(const BsrInstallParams &p) {
+  const uint64_t total = (uint64_t)p.n_chunks * p.n_tiles;
+  const uint64_t want = (uint64_t)kSmCount * 8;
+  return (uint32_t)(total < want ? total : want);
+}
+
+int launch_install(bsr_ctx *c, const BsrInstallParams &p, cudaStream_t s) {
+  bsr_install_vec_kernel<kInstallThreads, kInstallUnroll>
+      <<<install_grid(p), kInstallThreads, 0, s>>>(p);
+  CU(c, cudaGetLastError());
+  c->st.kernel_launches++;
+  c->st.install_launches++;
+  return BSR_OK;
+}
+
+// ---- filler threads: tier object -> pinned slot -------------------------------------------------
+void filler_main(bsr_ctx *c) {
+  for (;;) {
+    uint32_t s;
+    bsr_req *req;
+    {
+      std::unique_lock<std::mutex> lk(c->fill_mu);
+      c->fill_cv.wait(lk, [&] {
+        return c->fill_shutdown || (c->cur_req && c->fill_next < c->fill_admitted);
+      });
+      if (c->fill_shutdown) return;
+      s = c->fill_next++;
+      req = c->cur_req;
+      c->fill_active++;
+    }
+    const uint32_t R = c->cfg.n_ranks, W = c->cfg.window_chunks;
+    const uint32_t i = s / R, r = s % R;
+    int state = 1;
+    TierObj obj{};
+    if (!c->fill_abort.load(std::memory_order_acquire)) {
+      bool found = false;
+      {
+        std::lock_guard<std::mutex> g(c->mu);
+        auto it = c->tier[r].find(req->keys[i]);
+        if (it != c->tier[r].end()) {
+          obj = it->second;
+          found = true;
+        }
+      }
+      const Inject inj = c->inject;
+      const bool hit = inj.kind != BSR_INJECT_NONE && inj.rank == r && inj.chunk == i;
+      if (!found) {
+        state = BSR_ERR_MISSING;
+      } else if (hit && inj.kind == BSR_INJECT_FILL_ERROR) {
+        state = BSR_ERR_TRANSFER;
+      } else if (hit && inj.kind == BSR_INJECT_FILL_STALL) {
+        while (!c->fill_abort.load(std::memory_order_acquire) &&
+               Clock::now() < c->fill_deadline + std::chrono::seconds(5))
+          std::this_thread::sleep_for(std::chrono::milliseconds(1));
+        state = BSR_ERR_TIMEOUT;
+      } else if (obj.loc == BSR_LOC_HOST) {
+        uint8_t *slot = c->ring[r] + (size_t)(i % W) * c->slot_bytes;
+        memcpy(slot, obj.data, obj.len);
+        if (hit && inj.kind == BSR_INJECT_CORRUPT_SLOT && inj.group < c->G) {
+          const uint64_t words = c->seg_bytes[inj.group] / 4;
+          uint32_t *w = reinterpret_cast<uint32_t *>(slot + c->seg_begin[inj.group]);
+          w[inj.seed % words] ^= (uint32_t)(0x80000000u >> (inj.seed % 31));
+        }
+      }
+    }
+    (*c->task_obj)[s] = obj;
+    (*c->task_state)[s].store(state, std::memory_order_release);
+    {
+      std::lock_guard<std::mutex> lk(c->fill_mu);
+      c->fill_active--;
+    }
+    c->fill_cv.notify_all();
+  }
+}
+
+int ensure_ring(bsr_ctx *c) {
+  if (c->ring_ready) return BSR_OK;
+  const uint32_t R = c->cfg.n_ranks, W = c->cfg.window_chunks, D = c->cfg.dev_staging_depth;
+  for (uint32_t r = 0; r < R; ++r) {
+    if (cudaHostAlloc((void **)&c->ring[r], (size_t)W * c->slot_bytes, cudaHostAllocDefault) !=
+        cudaSuccess) {
+      cudaGetLastError();
+      return fail(c, BSR_ERR_NOMEM, "pinned ring of %u x %llu bytes", W,
+                  (unsigned long long)c->slot_bytes);
+    }
+    c->st.ring_bytes_allocated[r] = (uint64_t)W * c->slot_bytes;
+    if (cudaMalloc((void **)&c->dstage[r], (size_t)D * c->chunk_bytes) != cudaSuccess) {
+      cudaGetLastError();
+      return fail(c, BSR_ERR_NOMEM, "device staging of %u x %llu bytes", D,
+                  (unsigned long long)c->chunk_bytes);
+    }
+    c->st.dev_aux_bytes += (uint64_t)D * c->chunk_bytes;
+  }
+  c->ev_h2d.resize(R * D);
+  c->ev_inst.resize(R * D);
+  c->ev_start.resize(R * D);
+  for (uint32_t k = 0; k < R * D; ++k) {
+    CU(c, cudaEventCreateWithFlags(&c->ev_h2d[k], cudaEventDisableTiming));
+    CU(c, cudaEventCreate(&c->ev_inst[k]));
+    CU(c, cudaEventCreate(&c->ev_start[k]));
+  }
+  for (uint32_t k = 0; k < c->cfg.load_concurrency; ++k) c->fillers.emplace_back(filler_main, c);
+  c->ring_ready = true;
+  return BSR_OK;
+}
+
+void clear_request_state(bsr_req *q) {
+  std::fill(q->bitmap.begin(), q->bitmap.end(), 0ull);
+  q->restored = false;
+}
+
+void invalidate_host(bsr_req *q) {
+  std::fill(q->bitmap.begin(), q->bitmap.end(), 0ull);
+  q->failed = true;
+}
+
+// Reads the verdicts of chunk i of rank r after its install event completed.
+int harvest(bsr_ctx *c, bsr_req *q, uint32_t r, uint32_t i) {
+  int rc = BSR_OK;
+  for (uint32_t g = 0; g < c->G; ++g) {
+    const size_t o = ((size_t)r * c->G + g) * q->n_adv + i;
+    const uint32_t v = reinterpret_cast<volatile uint32_t *>(q->h_verdict)[o];
+    if (v == 1u)
+      q->bitmap[((size_t)r * c->G + g) * q->words + i / 64] |= 1ull << (i % 64);
+    else
+      rc = (v == 2u) ? BSR_ERR_CHECKSUM : BSR_ERR_TRANSFER;
+  }
+  if (rc == BSR_OK) c->st.bytes_installed[r] += c->chunk_bytes;
+  return rc;
+}
+
+int wait_event_deadline(bsr_ctx *c, cudaEvent_t ev, Clock::time_point deadline) {
+  for (;;) {
+    cudaError_t e = cudaEventQuery(ev);
+    if (e == cudaSuccess) return BSR_OK;
+    if (e != cudaErrorNotReady) return fail(c, BSR_ERR_CUDA, "event: %s", cudaGetErrorString(e));
+    if (Clock::now() > deadline) return BSR_ERR_TIMEOUT;
+    std::this_thread::yield();
+  }
+}
+
+// ---- restore when every advertised chunk already lives in device memory --------------------------
+int restore_resident(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_point deadline,
+                     const std::vector<TierObj> &objs) {
+  const uint32_t R = c->cfg.n_ranks, W = c->cfg.window_chunks, N = q->n_adv;
+  const uint32_t per_launch = BSR_K_MAX_BATCH / R ? BSR_K_MAX_BATCH / R : 1;
+  std::vector<std::pair<cudaEvent_t, cudaEvent_t>> timing;
+  int rc = BSR_OK;
+  cudaEvent_t done;
+  CU(c, cudaEventCreateWithFlags(&done, cudaEventDisableTiming));
+  for (uint32_t w0 = 0; w0 < N && rc == BSR_OK; w0 += W) {
+    const uint32_t w1 = (w0 + W < N) ? w0 + W : N;
+    c->st.windows++;
+    for (uint32_t b0 = w0; b0 < w1 && rc == BSR_OK; b0 += per_launch) {
+      const uint32_t b1 = (b0 + per_launch < w1) ? b0 + per_launch : w1;
+      BsrInstallParams p{};
+      fill_params(c, p, (uint32_t)(c->launch_seq++ % kLaunchSlots));
+      p.n_adv = N;
+      p.scatter = 1;
+      p.tables = q->d_table_ptrs;
+      p.ck_out = q->d_ck;
+      p.verdict = q->d_verdict;
+      for (uint32_t i = b0; i < b1; ++i)
+        for (uint32_t r = 0; r < R; ++r) {
+          BsrChunkDesc &d = p.chunk[p.n_chunks++];
+          const TierObj &o = objs[(size_t)i * R + r];
+          d.src = o.data;
+          d.chunk = i;
+          d.rank = r;
+          for (uint32_t g = 0; g < c->G; ++g) d.expect[g] = o.ck[g];
+        }
+      cudaEvent_t e0 = nullptr, e1 = nullptr;
+      if (c->cfg.time_kernels) {
+        CU(c, cudaEventCreate(&e0));
+        CU(c, cudaEventCreate(&e1));
+        CU(c, cudaEventRecord(e0, stream));
+      }
+      rc = launch_install(c, p, stream);
+      if (c->cfg.time_kernels) {
+        CU(c, cudaEventRecord(e1, stream));
+        timing.emplace_back(e0, e1);
+      }
+    }
+  }
+  CU(c, cudaEventRecord(done, stream));
+  int wrc = wait_event_deadline(c, done, deadline);
+  if (wrc == BSR_ERR_TIMEOUT) {  // kernels are finite: let them finish, then report
+    cudaStreamSynchronize(stream);
+  }
+  cudaEventDestroy(done);
+  for (auto &pr : timing) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, pr.first, pr.second) == cudaSuccess) c->st.install_kernel_ms += ms;
+    cudaEventDestroy(pr.first);
+    cudaEventDestroy(pr.second);
+  }
+  if (rc == BSR_OK) rc = wrc;
+  if (rc != BSR_OK) return rc;
+  for (uint32_t i = 0; i < N; ++i)
+    for (uint32_t r = 0; r < R; ++r) {
+      const int h = harvest(c, q, r, i);
+      if (h != BSR_OK && rc == BSR_OK) rc = h;
+    }
+  return rc;
+}
+
+// ---- restore through the pinned ring --------------------------------------------------------------
+int restore_ring(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_point deadline) {
+  int rc = ensure_ring(c);
+  if (rc != BSR_OK) return rc;
+  const uint32_t R = c->cfg.n_ranks, W = c->cfg.window_chunks, D = c->cfg.dev_staging_depth;
+  const uint32_t N = q->n_adv, total = N * R;
+  std::vector<std::atomic<int>> state(total);
+  for (auto &s : state) s.store(0, std::memory_order_relaxed);
+  std::vector<TierObj> objs(total);
+  {
+    std::lock_guard<std::mutex> lk(c->fill_mu);
+    c->cur_req = q;
+    c->fill_total = total;
+    c->fill_admitted = 0;
+    c->fill_next = 0;
+    c->fill_abort.store(false);
+    c->fill_deadline = deadline;
+    c->task_state = &state;
+    c->task_obj = &objs;
+  }
+  uint32_t admitted = 0, submitted = 0, reaped = 0;
+  uint32_t released[BSR_MAX_RANKS] = {};
+  for (uint32_t r = 0; r < R; ++r) c->live[r] = 0;
+  bool stop = false;  // a failure was seen: admit and submit nothing more, drain
+
+  auto first_error = [&](int code) {
+    if (rc == BSR_OK) rc = code;
+    stop = true;
+    c->fill_abort.store(true, std::memory_order_release);
+  };
+
+  while (true) {
+    bool progress = false;
+    // admit: chunk i of rank r enters the window as soon as slot i mod W is free (Eq. 3)
+    if (!stop) {
+      uint32_t n_new = 0;
+      while (admitted < total) {
+        const uint32_t i = admitted / R, r = admitted % R;
+        if (i - released[r] >= W) break;
+        if (i % W == 0 && r == 0) c->st.windows++;
+        c->live[r]++;
+        const uint64_t bytes = c->live[r] * c->slot_bytes;
+        if (bytes > c->st.peak_staging_bytes[r]) c->st.peak_staging_bytes[r] = bytes;
+        ++admitted;
+        ++n_new;
+      }
+      if (n_new) {
+        {
+          std::lock_guard<std::mutex> lk(c->fill_mu);
+          c->fill_admitted = admitted;
+        }
+        c->fill_cv.notify_all();
+        progress = true;
+      }
+    }
+    // reap, in order: observe the install of the oldest chunk in flight, release its slot
+    while (reaped < submitted) {
+      const uint32_t i = reaped / R, r = reaped % R, k = r * D + i % D;
+      cudaError_t e = cudaEventQuery(c->ev_inst[k]);
+      if (e == cudaErrorNotReady) break;
+      if (e != cudaSuccess) {
+        first_error(fail(c, BSR_ERR_CUDA, "install event: %s", cudaGetErrorString(e)));
+        reaped = submitted;  // the context is unusable; nothing more can be observed
+        break;
+      }
+      if (c->cfg.time_kernels) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, c->ev_start[k], c->ev_inst[k]) == cudaSuccess)
+          c->st.install_kernel_ms += ms;
+      }
+      const int h = harvest(c, q, r, i);
+      if (h != BSR_OK) first_error(h);
+      c->live[r]--;
+      released[r] = i + 1;
+      ++reaped;
+      progress = true;
+    }
+    // submit, in order: slot -> device staging on the copy stream, then the install kernel
+    while (!stop && submitted < admitted && submitted - reaped < R * D) {
+      const int stt = state[submitted].load(std::memory_order_acquire);
+      if (stt == 0) break;
+      if (stt < 0) {
+        first_error(stt);
+        break;
+      }
+      const uint32_t i = submitted / R, r = submitted % R, d = i % D, k = r * D + d;
+      const TierObj &o = objs[submitted];
+      uint8_t *stage = c->dstage[r] + (size_t)d * c->chunk_bytes;
+      const uint8_t *from = (o.loc == BSR_LOC_HOST) ? c->ring[r] + (size_t)(i % W) * c->slot_bytes
+                                                    : o.data;
+      cudaError_t e = cudaStreamWaitEvent(c->copy_stream, c->ev_inst[k], 0);
+      if (e == cudaSuccess)
+        e = cudaMemcpyAsync(stage, from, c->chunk_bytes, cudaMemcpyDefault, c->copy_stream);
+      if (e == cudaSuccess) e = cudaEventRecord(c->ev_h2d[k], c->copy_stream);
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, c->ev_h2d[k], 0);
+      if (e == cudaSuccess && c->cfg.time_kernels) e = cudaEventRecord(c->ev_start[k], stream);
+      if (e != cudaSuccess) {
+        first_error(fail(c, BSR_ERR_TRANSFER, "copy submit: %s", cudaGetErrorString(e)));
+        break;
+      }
+      c->st.h2d_copies++;
+      c->st.bytes_filled[r] += (o.loc == BSR_LOC_HOST) ? c->chunk_bytes : 0;
+      c->st.bytes_h2d[r] += c->chunk_bytes;
+      BsrInstallParams p{};
+      fill_params(c, p, (uint32_t)(c->launch_seq++ % kLaunchSlots));
+      p.n_adv = N;
+      p.scatter = 1;
+      p.tables = q->d_table_ptrs;
+      p.ck_out = q->d_ck;
+      p.verdict = q->d_verdict;
+      p.n_chunks = 1;
+      p.chunk[0].src = stage;
+      p.chunk[0].chunk = i;
+      p.chunk[0].rank = r;
+      for (uint32_t g = 0; g < c->G; ++g) p.chunk[0].expect[g] = o.ck[g];
+      const int lrc = launch_install(c, p, stream);
+      e = cudaEventRecord(c->ev_inst[k], stream);
+      if (lrc != BSR_OK || e != cudaSuccess) {
+        first_error(lrc != BSR_OK ? lrc : fail(c, BSR_ERR_CUDA, "record: %s", cudaGetErrorString(e)));
+        break;
+      }
+      ++submitted;
+      progress = true;
+    }
+    if (reaped == submitted && (stop || reaped == total)) break;
+    if (!progress) {
+      if (Clock::now() > deadline) {
+        first_error(BSR_ERR_TIMEOUT);
+        // copies and kernels already queued are finite: wait for them, then reap
+        cudaStreamSynchronize(c->copy_stream);
+        cudaStreamSynchronize(stream);
+        continue;
+      }
+      std::this_thread::yield();
+    }
+  }
+  // quiesce the fillers: nothing of this request may be touched after return
+  c->fill_abort.store(true, std::memory_order_release);
+  {
+    std::unique_lock<std::mutex> lk(c->fill_mu);
+    c->fill_admitted = c->fill_next;  // hand out no further task
+    c->fill_cv.wait(lk, [&] { return c->fill_active == 0; });
+    c->cur_req = nullptr;
+    c->task_state = nullptr;
+    c->task_obj = nullptr;
+  }
+  for (uint32_t r = 0; r < R; ++r) c->live[r] = 0;
+  return rc;
+}
+
+}  // namespace
+
+// =================================================================================================
+// C interface
+// =================================================================================================
+extern "C" {
+
+int bsr_ctx_create(const bsr_config *cfg, bsr_ctx **out) {
+  if (!cfg || !out) return BSR_ERR_INVALID;
+  if (cfg->window_chunks == 0 || cfg->n_ranks == 0 || cfg->n_ranks > BSR_MAX_RANKS ||
+      cfg->chunk_tokens != BSR_CHUNK_TOKENS)
+    return BSR_ERR_INVALID;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || cfg->device < 0 || cfg->device >= ndev) {
+    cudaGetLastError();
+    return BSR_ERR_CUDA;
+  }
+  bsr_ctx *c = new (std::nothrow) bsr_ctx();
+  if (!c) return BSR_ERR_NOMEM;
+  c->cfg = *cfg;
+  if (c->cfg.load_concurrency == 0) c->cfg.load_concurrency = 4;
+  if (c->cfg.load_concurrency > 64) c->cfg.load_concurrency = 64;
+  if (c->cfg.dev_staging_depth == 0) c->cfg.dev_staging_depth = 4;
+  if (c->cfg.dev_staging_depth > 16) c->cfg.dev_staging_depth = 16;
+  if (c->cfg.timeout_ms == 0) c->cfg.timeout_ms = 30000;
+  if (c->cfg.slot_align == 0) c->cfg.slot_align = 4096;
+  const size_t acc_bytes = (size_t)kLaunchSlots * BSR_K_MAX_BATCH * BSR_K_MAX_GROUPS * 8;
+  const size_t cnt_bytes = (kLaunchSlots + 2) * sizeof(unsigned int);
+  bool ok = cudaSetDevice(cfg->device) == cudaSuccess &&
+            cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaStreamCreateWithFlags(&c->own_stream, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaMalloc(&c->d_acc, acc_bytes) == cudaSuccess &&
+            cudaMalloc(&c->d_counters, cnt_bytes) == cudaSuccess &&
+            cudaMemset(c->d_acc, 0, acc_bytes) == cudaSuccess &&
+            cudaMemset(c->d_counters, 0, cnt_bytes) == cudaSuccess &&
+            cudaDeviceSynchronize() == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    bsr_ctx_destroy(c);
+    return BSR_ERR_CUDA;
+  }
+  c->st.dev_aux_bytes = acc_bytes + cnt_bytes;
+  *out = c;
+  return BSR_OK;
+}
+
+int bsr_ctx_destroy(bsr_ctx *c) {
+  if (!c) return BSR_ERR_INVALID;
+  cudaSetDevice(c->cfg.device);
+  {
+    std::lock_guard<std::mutex> lk(c->fill_mu);
+    c->fill_shutdown = true;
+  }
+  c->fill_cv.notify_all();
+  for (auto &t : c->fillers) t.join();
+  cudaDeviceSynchronize();
+  for (uint32_t r = 0; r < BSR_MAX_RANKS; ++r) {
+    if (c->ring[r]) cudaFreeHost(c->ring[r]);
+    if (c->dstage[r]) cudaFree(c->dstage[r]);
+  }
+  for (auto e : c->ev_h2d) cudaEventDestroy(e);
+  for (auto e : c->ev_inst) cudaEventDestroy(e);
+  for (auto e : c->ev_start) cudaEventDestroy(e);
+  cudaFree(c->d_tiles);
+  cudaFree(c->d_tensor_base);
+  cudaFree(c->d_tensor_group);
+  cudaFree(c->d_tensor_run);
+  cudaFree(c->d_put_stage);
+  if (c->h_put_ck) cudaFreeHost(c->h_put_ck);
+  if (c->h_put_verdict) cudaFreeHost(c->h_put_verdict);
+  cudaFree(c->d_acc);
+  cudaFree(c->d_counters);
+  cudaFree(c->d_tok);
+  cudaFree(c->d_digests);
+  cudaFree(c->d_keys);
+  if (c->h_keys) cudaFreeHost(c->h_keys);
+  if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+  if (c->own_stream) cudaStreamDestroy(c->own_stream);
+  cudaGetLastError();
+  delete c;
+  return BSR_OK;
+}
+
+const char *bsr_last_error(bsr_ctx *c) { return c ? c->err.c_str() : "null context"; }
+
+int bsr_register(bsr_ctx *c, uint32_t rank, const bsr_group_desc *groups, uint32_t n_groups,
+                 const bsr_tensor_desc *tensors, uint32_t n_tensors) {
+  if (!c || !groups || !tensors) return BSR_ERR_INVALID;
+  if (rank >= c->cfg.n_ranks || n_groups == 0 || n_groups > BSR_MAX_GROUPS || n_tensors == 0 ||
+      n_tensors > 65535)
+    return fail(c, BSR_ERR_INVALID, "register: rank/groups/tensors out of range");
+  if (c->finalized) return fail(c, BSR_ERR_STATE, "register after the registration was used");
+  for (uint32_t g = 0; g < n_groups; ++g) {
+    const uint32_t B = groups[g].block_tokens;
+    if (B == 0 || BSR_CHUNK_TOKENS % B || BSR_CHUNK_TOKENS / B > 255 || groups[g].num_phys_blocks == 0)
+      return fail(c, BSR_ERR_INVALID, "group %u: block_tokens must divide 256", g);
+  }
+  uint32_t prev_group = 0;
+  uint64_t per_token = 0;
+  for (uint32_t l = 0; l < n_tensors; ++l) {
+    const bsr_tensor_desc &t = tensors[l];
+    if (t.group >= n_groups || t.group < prev_group)
+      return fail(c, BSR_ERR_INVALID, "tensor %u: tensors must be listed group-major", l);
+    prev_group = t.group;
+    if (t.bytes_per_token == 0 || t.bytes_per_token % 16)
+      return fail(c, BSR_ERR_ALIGN, "tensor %u: bytes_per_token must be a multiple of 16", l);
+    if (!t.dev_base || (reinterpret_cast<uintptr_t>(t.dev_base) & 15u))
+      return fail(c, BSR_ERR_ALIGN, "tensor %u: dev_base must be 16-byte aligned", l);
+    per_token += t.bytes_per_token;
+  }
+  if (per_token * BSR_CHUNK_TOKENS >= (1ull << 32))
+    return fail(c, BSR_ERR_INVALID, "chunk larger than 4 GiB");
+  std::lock_guard<std::mutex> lk(c->mu);
+  const bool first = (c->L == 0);
+  if (first) {
+    c->G = n_groups;
+    c->L = n_tensors;
+    c->groups.assign(groups, groups + n_groups);
+    c->tensors.resize(n_tensors);
+    uint64_t off = 0;
+    for (uint32_t g = 0; g < n_groups; ++g) c->seg_begin[g] = c->seg_bytes[g] = 0;
+    bool seen[BSR_MAX_GROUPS] = {};
+    for (uint32_t l = 0; l < n_tensors; ++l) {
+      c->tensors[l].group = tensors[l].group;
+      c->tensors[l].bytes_per_token = tensors[l].bytes_per_token;
+      const uint64_t sz = (uint64_t)BSR_CHUNK_TOKENS * tensors[l].bytes_per_token;
+      if (!seen[tensors[l].group]) {
+        seen[tensors[l].group] = true;
+        c->seg_begin[tensors[l].group] = off;
+      }
+      c->seg_bytes[tensors[l].group] += sz;
+      off += sz;
+    }
+    c->chunk_bytes = off;
+    c->slot_bytes = round_up(off, c->cfg.slot_align);
+    c->st.slot_bytes = c->slot_bytes;
+  } else {
+    bool same = (n_groups == c->G && n_tensors == c->L);
+    for (uint32_t g = 0; same && g < n_groups; ++g)
+      same = groups[g].block_tokens == c->groups[g].block_tokens &&
+             groups[g].num_phys_blocks == c->groups[g].num_phys_blocks;
+    for (uint32_t l = 0; same && l < n_tensors; ++l)
+      same = tensors[l].group == c->tensors[l].group &&
+             tensors[l].bytes_per_token == c->tensors[l].bytes_per_token;
+    if (!same) {
+      c->err = "register: every rank must register the same geometry";
+      return BSR_ERR_INVALID;
+    }
+  }
+  for (uint32_t l = 0; l < n_tensors; ++l)
+    c->tensors[l].base[rank] = reinterpret_cast<uint64_t>(tensors[l].dev_base);
+  c->rank_registered[rank] = true;
+  return BSR_OK;
+}
+
+int bsr_chunk_bytes(bsr_ctx *c, uint64_t *chunk_bytes, uint64_t *slot_bytes) {
+  if (!c) return BSR_ERR_INVALID;
+  if (c->L == 0) return fail(c, BSR_ERR_STATE, "no registration");
+  if (chunk_bytes) *chunk_bytes = c->chunk_bytes;
+  if (slot_bytes) *slot_bytes = c->slot_bytes;
+  return BSR_OK;
+}
+
+int bsr_tier_put(bsr_ctx *c, uint32_t rank, uint64_t key, const void *data, size_t len,
+                 const uint64_t *group_ck, int location) {
+  if (!c || !data) return BSR_ERR_INVALID;
+  if (rank >= c->cfg.n_ranks || (location != BSR_LOC_HOST && location != BSR_LOC_DEVICE))
+    return fail(c, BSR_ERR_INVALID, "tier_put: bad rank or location");
+  if (c->L == 0) return fail(c, BSR_ERR_STATE, "tier_put before registration");
+  if (len != c->chunk_bytes)
+    return fail(c, BSR_ERR_INVALID, "tier_put: len %zu != chunk bytes %llu", len,
+                (unsigned long long)c->chunk_bytes);
+  if (location == BSR_LOC_DEVICE && (reinterpret_cast<uintptr_t>(data) & 15u))
+    return fail(c, BSR_ERR_ALIGN, "tier_put: device object must be 16-byte aligned");
+  TierObj o{};
+  o.data = static_cast<const uint8_t *>(data);
+  o.len = len;
+  o.loc = location;
+  if (group_ck) {
+    for (uint32_t g = 0; g < c->G; ++g) o.ck[g] = group_ck[g];
+  } else {
+    // store path: compute the group checksums on the GPU with the install kernel's sum stage
+    std::lock_guard<std::mutex> rl(c->restore_mu);
+    CU(c, cudaSetDevice(c->cfg.device));
+    int rc = finalize_registration(c);
+    if (rc != BSR_OK) return rc;
+    if (!c->h_put_ck) {
+      CU(c, cudaHostAlloc((void **)&c->h_put_ck, BSR_MAX_GROUPS * 8, cudaHostAllocMapped));
+      CU(c, cudaHostAlloc((void **)&c->h_put_verdict, BSR_MAX_GROUPS * 4, cudaHostAllocMapped));
+      CU(c, cudaHostGetDevicePointer((void **)&c->d_put_ck, c->h_put_ck, 0));
+      CU(c, cudaHostGetDevicePointer((void **)&c->d_put_verdict, c->h_put_verdict, 0));
+    }
+    const uint8_t *src = o.data;
+    if (location == BSR_LOC_HOST) {
+      if (!c->d_put_stage) CU(c, cudaMalloc((void **)&c->d_put_stage, c->chunk_bytes));
+      CU(c, cudaMemcpyAsync(c->d_put_stage, data, len, cudaMemcpyHostToDevice, c->own_stream));
+      src = c->d_put_stage;
+    }
+    BsrInstallParams p{};
+    fill_params(c, p, (uint32_t)(c->launch_seq++ % kLaunchSlots));
+    p.n_adv = 1;
+    p.scatter = 0;
+    p.ck_out = c->d_put_ck;
+    p.verdict = c->d_put_verdict;
+    p.n_chunks = 1;
+    p.chunk[0].src = src;
+    rc = launch_install(c, p, c->own_stream);
+    if (rc != BSR_OK) return rc;
+    CU(c, cudaStreamSynchronize(c->own_stream));
+    for (uint32_t g = 0; g < c->G; ++g) o.ck[g] = c->h_put_ck[g];
+  }
+  std::lock_guard<std::mutex> lk(c->mu);
+  c->tier[rank][key] = o;
+  return BSR_OK;
+}
+
+int bsr_tier_remove(bsr_ctx *c, uint32_t rank, uint64_t key) {
+  if (!c || rank >= c->cfg.n_ranks) return BSR_ERR_INVALID;
+  std::lock_guard<std::mutex> lk(c->mu);
+  c->tier[rank].erase(key);
+  return BSR_OK;
+}
+
+int bsr_tier_checksums(bsr_ctx *c, uint32_t rank, uint64_t key, uint64_t *out) {
+  if (!c || !out || rank >= c->cfg.n_ranks) return BSR_ERR_INVALID;
+  std::lock_guard<std::mutex> lk(c->mu);
+  auto it = c->tier[rank].find(key);
+  if (it == c->tier[rank].end()) return BSR_ERR_MISSING;
+  for (uint32_t g = 0; g < c->G; ++g) out[g] = it->second.ck[g];
+  return BSR_OK;
+}
+
+int bsr_probe(bsr_ctx *c, const int32_t *tok, size_t n_tok, int tok_on_device, uint64_t salt,
+              uint64_t *keys_out, uint64_t *hit_bitmap_out, uint32_t *n_hit_chunks) {
+  if (!c || (!tok && n_tok) || !n_hit_chunks) return BSR_ERR_INVALID;
+  const size_t N = n_tok / BSR_CHUNK_TOKENS;
+  if (N > (1u << 24)) return fail(c, BSR_ERR_INVALID, "probe: more than 2^24 chunks");
+  if (tok_on_device && (reinterpret_cast<uintptr_t>(tok) & 15u))
+    return fail(c, BSR_ERR_ALIGN, "probe: device token ids must be 16-byte aligned");
+  if (N == 0) {
+    *n_hit_chunks = 0;
+    return BSR_OK;
+  }
+  std::lock_guard<std::mutex> rl(c->restore_mu);  // probe scratch is per context
+  CU(c, cudaSetDevice(c->cfg.device));
+  if (N > c->probe_cap_chunks) {
+    cudaFree(c->d_tok);
+    cudaFree(c->d_digests);
+    cudaFree(c->d_keys);
+    if (c->h_keys) cudaFreeHost(c->h_keys);
+    c->d_tok = nullptr;
+    c->d_digests = c->d_keys = c->h_keys = nullptr;
+    c->probe_cap_chunks = 0;
+    const size_t cap = round_up(N, 1024);
+    CU(c, cudaMalloc((void **)&c->d_tok, cap * BSR_CHUNK_TOKENS * 4));
+    CU(c, cudaMalloc((void **)&c->d_digests, cap * 8));
+    CU(c, cudaMalloc((void **)&c->d_keys, cap * 8));
+    CU(c, cudaHostAlloc((void **)&c->h_keys, cap * 8, cudaHostAllocDefault));
+    c->probe_cap_chunks = cap;
+  }
+  const int32_t *d_tok = tok;
+  cudaStream_t s = c->own_stream;
+  if (!tok_on_device) {
+    CU(c, cudaMemcpyAsync(c->d_tok, tok, N * BSR_CHUNK_TOKENS * 4, cudaMemcpyHostToDevice, s));
+    d_tok = c->d_tok;
+  }
+  // k_-1 = mix64(salt ^ mix64(reg_id)); a scalar, computed once per call
+  auto mix = [](uint64_t x) {
+    x += BSR_K_PHI;
+    x = (x ^ (x >> 32)) * BSR_K_PHI;
+    x = (x ^ (x >> 29)) * BSR_K_PHI;
+    return x ^ (x >> 32);
+  };
+  const uint64_t k_init = mix(salt ^ mix(c->cfg.reg_id));
+  const uint32_t per_block = BSR_K_PROBE_THREADS / 32;
+  const uint32_t grid = (uint32_t)((N + per_block - 1) / per_block);
+  bsr_probe_kernel<<<grid, BSR_K_PROBE_THREADS, 0, s>>>(d_tok, (uint32_t)N, salt, k_init,
+                                                        c->d_digests, c->d_counters + kLaunchSlots,
+                                                        c->d_keys);
+  CU(c, cudaGetLastError());
+  c->st.kernel_launches++;
+  CU(c, cudaMemcpyAsync(c->h_keys, c->d_keys, N * 8, cudaMemcpyDeviceToHost, s));
+  CU(c, cudaStreamSynchronize(s));
+  // index lookup: keys only; no payload byte is read, nothing is pinned or referenced afterwards
+  uint32_t n_hit = 0;
+  bool prefix = true;
+  if (hit_bitmap_out) memset(hit_bitmap_out, 0, (N + 63) / 64 * 8);
+  {
+    std::lock_guard<std::mutex> lk(c->mu);
+    for (size_t i = 0; i < N; ++i) {
+      bool hit = true;
+      for (uint32_t r = 0; r < c->cfg.n_ranks && hit; ++r)
+        hit = c->tier[r].find(c->h_keys[i]) != c->tier[r].end();
+      if (hit && hit_bitmap_out) hit_bitmap_out[i / 64] |= 1ull << (i % 64);
+      if (!hit) prefix = false;
+      if (prefix) ++n_hit;
+    }
+  }
+  if (keys_out) memcpy(keys_out, c->h_keys, N * 8);
+  *n_hit_chunks = n_hit;
+  return BSR_OK;
+}
+
+int bsr_req_create(bsr_ctx *c, const uint64_t *keys, uint32_t n_adv, const int32_t *const *tables,
+                   bsr_req **out) {
+  if (!c || !out || (n_adv && (!keys || !tables))) return BSR_ERR_INVALID;
+  {
+    std::lock_guard<std::mutex> rl(c->restore_mu);
+    CU(c, cudaSetDevice(c->cfg.device));
+    int rc = finalize_registration(c);
+    if (rc != BSR_OK) return rc;
+  }
+  const uint32_t R = c->cfg.n_ranks, G = c->G;
+  bsr_req *q = new (std::nothrow) bsr_req();
+  if (!q) return BSR_ERR_NOMEM;
+  q->ctx = c;
+  q->n_adv = n_adv;
+  q->keys.assign(keys, keys + n_adv);
+  q->words = (n_adv + 63) / 64;
+  q->bitmap.assign((size_t)R * G * q->words, 0ull);
+  q->tables.resize((size_t)R * G);
+  size_t total_entries = 0;
+  for (uint32_t r = 0; r < R; ++r)
+    for (uint32_t g = 0; g < G; ++g) {
+      const size_t n = (size_t)n_adv * (BSR_CHUNK_TOKENS / c->groups[g].block_tokens);
+      const int32_t *t = tables[r * G + g];
+      if (n && !t) {
+        delete q;
+        return fail(c, BSR_ERR_INVALID, "req_create: null block table");
+      }
+      std::vector<bool> seen(c->groups[g].num_phys_blocks, false);
+      for (size_t j = 0; j < n; ++j) {
+        if (t[j] < 0 || (uint32_t)t[j] >= c->groups[g].num_phys_blocks || seen[t[j]]) {
+          delete q;
+          return fail(c, BSR_ERR_INVALID,
+                      "req_create: table (rank %u, group %u) entry %zu out of range or repeated", r,
+                      g, j);
+        }
+        seen[t[j]] = true;
+      }
+      q->tables[r * G + g].assign(t, t + n);
+      total_entries += n;
+    }
+  auto bail = [&](int code, const char *what) {
+    bsr_req_release(c, q);
+    return fail(c, code, "req_create: %s", what);
+  };
+  cudaSetDevice(c->cfg.device);
+  if (n_adv) {
+    if (cudaMalloc((void **)&q->d_tables, total_entries * 4) != cudaSuccess ||
+        cudaMalloc((void **)&q->d_table_ptrs, (size_t)R * G * sizeof(void *)) != cudaSuccess)
+      return bail(BSR_ERR_NOMEM, "device block tables");
+    std::vector<const int32_t *> ptrs((size_t)R * G);
+    size_t off = 0;
+    for (size_t k = 0; k < q->tables.size(); ++k) {
+      ptrs[k] = q->d_tables + off;
+      if (!q->tables[k].empty() &&
+          cudaMemcpy(q->d_tables + off, q->tables[k].data(), q->tables[k].size() * 4,
+                     cudaMemcpyHostToDevice) != cudaSuccess)
+        return bail(BSR_ERR_CUDA, "table upload");
+      off += q->tables[k].size();
+    }
+    if (cudaMemcpy(q->d_table_ptrs, ptrs.data(), ptrs.size() * sizeof(void *),
+                   cudaMemcpyHostToDevice) != cudaSuccess)
+      return bail(BSR_ERR_CUDA, "table pointer upload");
+    const size_t cells = (size_t)R * G * n_adv;
+    if (cudaHostAlloc((void **)&q->h_ck, cells * 8, cudaHostAllocMapped) != cudaSuccess ||
+        cudaHostAlloc((void **)&q->h_verdict, cells * 4, cudaHostAllocMapped) != cudaSuccess ||
+        cudaHostGetDevicePointer((void **)&q->d_ck, q->h_ck, 0) != cudaSuccess ||
+        cudaHostGetDevicePointer((void **)&q->d_verdict, q->h_verdict, 0) != cudaSuccess)
+      return bail(BSR_ERR_NOMEM, "status arrays");
+    memset(q->h_ck, 0, cells * 8);
+    memset(q->h_verdict, 0, cells * 4);
+  }
+  *out = q;
+  return BSR_OK;
+}
+
+int bsr_req_release(bsr_ctx *c, bsr_req *q) {
+  if (!c || !q || q->ctx != c) return BSR_ERR_INVALID;
+  std::lock_guard<std::mutex> rl(c->restore_mu);
+  cudaSetDevice(c->cfg.device);
+  cudaFree(q->d_tables);
+  cudaFree(q->d_table_ptrs);
+  if (q->h_ck) cudaFreeHost(q->h_ck);
+  if (q->h_verdict) cudaFreeHost(q->h_verdict);
+  cudaGetLastError();
+  delete q;
+  return BSR_OK;
+}
+
+int bsr_restore(bsr_ctx *c, bsr_req *q, void *cuda_stream) {
+  if (!c || !q || q->ctx != c) return BSR_ERR_INVALID;
+  std::lock_guard<std::mutex> rl(c->restore_mu);  // bounded-retrieve lock
+  const auto t0 = Clock::now();
+  const auto deadline = t0 + std::chrono::milliseconds(c->cfg.timeout_ms);
+  CU(c, cudaSetDevice(c->cfg.device));
+  cudaStream_t stream = cuda_stream ? static_cast<cudaStream_t>(cuda_stream) : c->own_stream;
+  clear_request_state(q);
+  q->failed = false;
+  const uint32_t R = c->cfg.n_ranks, N = q->n_adv;
+  if (N) {
+    const size_t cells = (size_t)R * c->G * N;
+    memset(q->h_ck, 0, cells * 8);
+    memset(q->h_verdict, 0, cells * 4);
+  }
+  int rc = BSR_OK;
+  if (N) {
+    // are all advertised chunks already in device memory?  (then no staging is needed at all)
+    std::vector<TierObj> objs((size_t)N * R);
+    bool all_device = true;
+    {
+      std::lock_guard<std::mutex> lk(c->mu);
+      for (uint32_t i = 0; i < N && all_device; ++i)
+        for (uint32_t r = 0; r < R; ++r) {
+          auto it = c->tier[r].find(q->keys[i]);
+          if (it == c->tier[r].end() || it->second.loc != BSR_LOC_DEVICE) {
+            all_device = false;
+            break;
+          }
+          objs[(size_t)i * R + r] = it->second;
+        }
+    }
+    rc = all_device ? restore_resident(c, q, stream, deadline, objs)
+                    : restore_ring(c, q, stream, deadline);
+  }
+  if (rc == BSR_OK)
+    q->restored = true;
+  else
+    invalidate_host(q);
+  c->inject.kind = BSR_INJECT_NONE;  // one shot
+  c->st.last_restore_ms = std::chrono::duration<double, std::milli>(Clock::now() - t0).count();
+  return rc;
+}
+
+int bsr_commit(bsr_ctx *c, bsr_req *q, uint32_t *exposed) {
+  if (!c || !q || q->ctx != c || !exposed) return BSR_ERR_INVALID;
+  std::lock_guard<std::mutex> rl(c->restore_mu);
+  bool all = q->restored && !q->failed;
+  const uint32_t R = c->cfg.n_ranks;
+  for (uint32_t rg = 0; all && rg < R * c->G; ++rg)
+    for (uint32_t w = 0; all && w < q->words; ++w) {
+      const uint32_t bits = (w + 1 < q->words || q->n_adv % 64 == 0) ? 64 : q->n_adv % 64;
+      const uint64_t want = bits == 64 ? ~0ull : ((1ull << bits) - 1);
+      all = q->bitmap[(size_t)rg * q->words + w] == want;
+    }
+  if (all) {
+    *exposed = q->n_adv;
+  } else {
+    invalidate_host(q);
+    *exposed = 0;
+  }
+  return BSR_OK;
+}
+
+int bsr_invalidate(bsr_ctx *c, bsr_req *q, unsigned flags) {
+  if (!c || !q || q->ctx != c) return BSR_ERR_INVALID;
+  std::lock_guard<std::mutex> rl(c->restore_mu);
+  invalidate_host(q);
+  if ((flags & BSR_SCRUB) && q->n_adv) {
+    CU(c, cudaSetDevice(c->cfg.device));
+    BsrScrubParams p{};
+    p.tensor_base = c->d_tensor_base;
+    p.tables = q->d_table_ptrs;
+    p.tensor_group = c->d_tensor_group;
+    p.tensor_run = c->d_tensor_run;
+    p.n_tensors = c->L;
+    p.n_groups = c->G;
+    p.n_adv = q->n_adv;
+    uint32_t max_logical = 0;
+    for (uint32_t g = 0; g < c->G; ++g) {
+      p.blocks_per_chunk[g] = BSR_CHUNK_TOKENS / c->groups[g].block_tokens;
+      const uint32_t n = q->n_adv * p.blocks_per_chunk[g];
+      if (n > max_logical) max_logical = n;
+    }
+    dim3 grid(max_logical < 1024 ? max_logical : 1024, c->cfg.n_ranks * c->L);
+    bsr_scrub_kernel<<<grid, 256, 0, c->own_stream>>>(p);
+    CU(c, cudaGetLastError());
+    c->st.kernel_launches++;
+    CU(c, cudaStreamSynchronize(c->own_stream));
+  }
+  return BSR_OK;
+}
+
+int bsr_req_bitmap(bsr_ctx *c, bsr_req *q, uint64_t *out, size_t words) {
+  if (!c || !q || q->ctx != c || (!out && words)) return BSR_ERR_INVALID;
+  if (words < q->bitmap.size()) return fail(c, BSR_ERR_INVALID, "bitmap buffer too small");
+  std::lock_guard<std::mutex> rl(c->restore_mu);
+  if (!q->bitmap.empty()) memcpy(out, q->bitmap.data(), q->bitmap.size() * 8);
+  return BSR_OK;
+}
+
+int bsr_req_checksums(bsr_ctx *c, bsr_req *q, uint64_t *out, size_t count) {
+  if (!c || !q || q->ctx != c || (!out && count)) return BSR_ERR_INVALID;
+  const size_t cells = (size_t)c->cfg.n_ranks * c->G * q->n_adv;
+  if (count < cells) return fail(c, BSR_ERR_INVALID, "checksum buffer too small");
+  std::lock_guard<std::mutex> rl(c->restore_mu);
+  if (cells) memcpy(out, q->h_ck, cells * 8);
+  return BSR_OK;
+}
+
+int bsr_get_stats(bsr_ctx *c, bsr_stats *out) {
+  if (!c || !out) return BSR_ERR_INVALID;
+  std::lock_guard<std::mutex> rl(c->restore_mu);
+  *out = c->st;
+  return BSR_OK;
+}
+
+int bsr_reset_stats(bsr_ctx *c) {
+  if (!c) return BSR_ERR_INVALID;
+  std::lock_guard<std::mutex> rl(c->restore_mu);
+  bsr_stats keep = c->st;
+  c->st = bsr_stats{};
+  c->st.slot_bytes = keep.slot_bytes;
+  c->st.dev_aux_bytes = keep.dev_aux_bytes;
+  for (uint32_t r = 0; r < BSR_MAX_RANKS; ++r)
+    c->st.ring_bytes_allocated[r] = keep.ring_bytes_allocated[r];
+  return BSR_OK;
+}
+
+int bsr_test_inject(bsr_ctx *c, int kind, uint32_t rank, uint32_t group, uint32_t chunk,
+                    uint64_t seed) {
+  if (!c || kind < BSR_INJECT_NONE || kind > BSR_INJECT_FILL_STALL) return BSR_ERR_INVALID;
+  std::lock_guard<std::mutex> rl(c->restore_mu);
+  c->inject.kind = kind;
+  c->inject.rank = rank;
+  c->inject.group = group;
+  c->inject.chunk = chunk;
+  c->inject.seed = seed;
+  return BSR_OK;
+}
+
+}  // extern "C"

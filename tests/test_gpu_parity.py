@@ -1,0 +1,257 @@
+"""CUDA path vs CPU oracle, element by element, through the C interface (needs a B200)."""
+import numpy as np
+import pytest
+
+from harness import Case, GpuSide, assert_paged_equal, run_oracle
+from oracle import bsr_oracle as O
+from paper_2608_17826_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _check_success(case, W, gpu, ora, n_adv):
+    B = gpu.B
+    st = gpu.stats()
+    slot = case.reg.slot_bytes
+    assert gpu.commit() == ora["exposed"] == n_adv
+    assert np.array_equal(gpu.bitmap(n_adv), ora["req"].bitmap())
+    assert_paged_equal(gpu, ora["paged"])
+    rc, cks = B.bsr_req_checksums(gpu.ctx, gpu.req, case.R, case.G, n_adv)
+    assert rc == B.BSR_OK
+    for r in range(case.R):
+        for i in range(n_adv):
+            assert [int(x) for x in cks[r, :, i]] == case.cks[(r, i)]
+    assert st.windows == ora["stats"].windows == -(-n_adv // W)
+    for r in range(case.R):
+        assert st.bytes_installed[r] == ora["stats"].bytes_installed[r] == n_adv * case.reg.chunk_bytes
+        if gpu.location == B.BSR_LOC_HOST:
+            assert st.peak_staging_bytes[r] == ora["stats"].peak_staging_bytes[r] == min(n_adv, W) * slot
+            assert st.bytes_filled[r] == st.bytes_h2d[r] == ora["stats"].bytes_filled[r]
+            assert st.ring_bytes_allocated[r] == W * slot
+        else:
+            assert st.peak_staging_bytes[r] == 0 and st.bytes_h2d[r] == 0
+    assert st.slot_bytes == slot
+    assert st.tier_bytes_read_by_probe == 0
+
+
+# ---------------------------------------------------------------- probe
+@pytest.mark.parametrize("N,tail,on_device", [(1, 0, False), (37, 100, False), (37, 100, True),
+                                              (2048, 0, True), (2051, 255, False)])
+def test_probe_keys_bitmap_prefix(N, tail, on_device):
+    layout = synth.tiny_layout()
+    present = (lambda r, i: i < 20 or i == 25 or (r == 1 and i == 20)) if N == 37 else (lambda r, i: i < 3)
+    case = Case(layout, 2, N, seed=101, present=present, tail_tokens=tail)
+    tiers = case.oracle_tiers()
+    keys, hit, n_hit = O.probe(case.tok, case.salt, case.reg_id, tiers)
+    with GpuSide(case, W=4) as gpu:
+        rc, k, bm, nh = gpu.probe(tok_on_device=on_device)
+        assert rc == gpu.B.BSR_OK
+        assert np.array_equal(k, keys)
+        assert np.array_equal(bm, O.pack_bits(hit))
+        assert nh == n_hit == min(N, 20 if N == 37 else 3)
+        st = gpu.stats()
+        assert st.tier_bytes_read_by_probe == 0 and max(st.peak_staging_bytes) == 0
+        # another salt: nothing reusable
+        rc, k2, _, nh2 = gpu.B.bsr_probe(gpu.ctx, case.tok, len(case.tok), case.salt + 1)
+        assert rc == gpu.B.BSR_OK and nh2 == 0 and not np.array_equal(k2, keys)
+
+
+def test_probe_fewer_than_one_chunk():
+    case = Case(synth.tiny_layout(), 1, 1, seed=102)
+    with GpuSide(case, W=2) as gpu:
+        rc, k, bm, nh = gpu.B.bsr_probe(gpu.ctx, case.tok[:200].copy(), 200, case.salt)
+        assert rc == gpu.B.BSR_OK and nh == 0 and len(k) == 0
+
+
+# ---------------------------------------------------------------- restore, success
+@pytest.mark.parametrize("layout_name,R,N,W,cfg", [
+    ("tiny", 1, 1, 1, {}),
+    ("tiny", 2, 5, 2, {}),
+    ("tiny", 2, 9, 4, dict(load_concurrency=1, dev_staging_depth=1)),
+    ("tiny", 2, 23, 8, dict(load_concurrency=8, dev_staging_depth=2)),
+    ("tiny", 3, 7, 64, {}),                      # W >= N: whole plan live at once
+    ("tiny", 2, 70, 3, dict(load_concurrency=3)),
+    ("hetero", 2, 6, 4, {}),
+    ("baseline", 1, 16, 4, {}),                  # the tiny single-rank configuration
+])
+def test_restore_matches_oracle(layout_name, R, N, W, cfg):
+    layout = {"tiny": synth.tiny_layout, "hetero": synth.hetero_layout,
+              "baseline": synth.baseline_layout}[layout_name]()
+    case = Case(layout, R, N, seed=200 + N)
+    ora = run_oracle(case, W)
+    assert ora["status"] == O.OK and ora["n_hit"] == N
+    with GpuSide(case, W, **cfg) as gpu:
+        rc, keys, bm, n_hit = gpu.probe()
+        assert rc == gpu.B.BSR_OK and n_hit == N and np.array_equal(keys, ora["keys"])
+        gpu.request(keys, n_hit)
+        assert gpu.restore() == gpu.B.BSR_OK, gpu.B.bsr_last_error(gpu.ctx)
+        _check_success(case, W, gpu, ora, N)
+        # a second restore of the same request is idempotent
+        gpu.B.bsr_reset_stats(gpu.ctx)
+        assert gpu.restore() == gpu.B.BSR_OK
+        _check_success(case, W, gpu, ora, N)
+
+
+@pytest.mark.parametrize("layout_name,R,N,W", [("tiny", 2, 11, 4), ("hetero", 2, 5, 2), ("baseline", 2, 6, 4)])
+def test_restore_from_device_resident_tier(layout_name, R, N, W):
+    layout = {"tiny": synth.tiny_layout, "hetero": synth.hetero_layout,
+              "baseline": synth.baseline_layout}[layout_name]()
+    case = Case(layout, R, N, seed=300 + N)
+    ora = run_oracle(case, W)
+    with GpuSide(case, W, location=1, time_kernels=True) as gpu:
+        rc, keys, bm, n_hit = gpu.probe()
+        gpu.request(keys, n_hit)
+        assert gpu.restore() == gpu.B.BSR_OK, gpu.B.bsr_last_error(gpu.ctx)
+        _check_success(case, W, gpu, ora, N)
+        assert gpu.stats().install_kernel_ms > 0
+
+
+def test_library_computed_checksums_equal_oracle():
+    for layout in (synth.tiny_layout(), synth.hetero_layout()):
+        case = Case(layout, 2, 3, seed=400)
+        for loc in (0, 1):
+            with GpuSide(case, 2, location=loc, compute_ck=True) as gpu:
+                for (r, i), want in case.cks.items():
+                    rc, got = gpu.B.bsr_tier_checksums(gpu.ctx, r, case.keys[i], case.G)
+                    assert rc == gpu.B.BSR_OK and [int(x) for x in got] == want
+
+
+def test_partial_hit_exposes_exactly_the_prefix():
+    case = Case(synth.tiny_layout(), 2, 20, seed=500, present=lambda r, i: i < 13 or i == 16)
+    ora = run_oracle(case, 4)
+    assert ora["n_hit"] == 13 and ora["exposed"] == 13
+    with GpuSide(case, 4) as gpu:
+        rc, keys, bm, n_hit = gpu.probe()
+        assert n_hit == 13 and np.array_equal(bm, O.pack_bits(ora["hit"]))
+        gpu.request(keys, n_hit)
+        assert gpu.restore() == gpu.B.BSR_OK
+        _check_success(case, 4, gpu, ora, 13)
+
+
+# ---------------------------------------------------------------- failures: fail closed
+def _check_failed(case, W, gpu, n_adv, want_rc, scrub_paged):
+    B = gpu.B
+    assert gpu.commit() == 0
+    assert (gpu.bitmap(n_adv) == 0).all()
+    st = gpu.stats()
+    assert 0 < max(st.peak_staging_bytes[: case.R]) <= W * case.reg.slot_bytes
+    assert B.bsr_invalidate(gpu.ctx, gpu.req, B.BSR_SCRUB) == B.BSR_OK
+    assert_paged_equal(gpu, scrub_paged)          # request blocks zero, every other block untouched
+    assert gpu.commit() == 0
+
+
+def _scrubbed_oracle(case, W, n_adv, mutate_tiers=None, fetch_fault=None):
+    tiers = case.oracle_tiers()
+    if mutate_tiers:
+        mutate_tiers(tiers)
+    ora = run_oracle(case, W, n_adv=n_adv, tiers=tiers, fetch_fault=fetch_fault)
+    assert ora["status"] != O.OK and ora["exposed"] == 0 and not ora["req"].valid.any()
+    O.invalidate(case.reg, ora["req"], ora["paged"], scrub=True)
+    return ora
+
+
+FAILURE_KINDS = ["corrupt_tier", "missing", "rank_asymmetric", "corrupt_slot", "fill_error", "fill_stall"]
+
+
+@pytest.mark.parametrize("kind", FAILURE_KINDS)
+def test_failures_expose_nothing(kind):
+    layout = synth.tiny_layout()
+    R, N, W = 2, 24, 4
+    case = Case(layout, R, N, seed=600)
+    r, g, i, frac = synth.fault_site(R, case.G, W, N, case=FAILURE_KINDS.index(kind), seed=7)
+    if kind == "rank_asymmetric":
+        r, g = 1, 1
+    cfg = dict(timeout_ms=1500) if kind == "fill_stall" else {}
+    with GpuSide(case, W, **cfg) as gpu:
+        B = gpu.B
+        rc, keys, bm, n_hit = gpu.probe()
+        assert n_hit == N
+        gpu.request(keys, N)
+        fetch_fault = None
+        mutate = None
+        want = None
+        if kind in ("corrupt_tier", "rank_asymmetric"):
+            lo, hi = case.reg.segment(g)
+            w = case.payload[(r, i)][lo:hi].view("<u4")
+            w[frac % len(w)] ^= np.uint32(1 << (frac % 32))      # tier bytes are caller-owned
+            want = B.BSR_ERR_CHECKSUM
+        elif kind == "missing":
+            assert B.bsr_tier_remove(gpu.ctx, r, case.keys[i]) == B.BSR_OK   # after probe
+            mutate = lambda tiers: tiers[r].remove(case.keys[i])
+            want = B.BSR_ERR_MISSING
+        elif kind == "corrupt_slot":
+            B.bsr_test_inject(gpu.ctx, B.BSR_INJECT_CORRUPT_SLOT, r, g, i, frac)
+            lo, hi = case.reg.segment(g)
+            def mutate(tiers, lo=lo, hi=hi):
+                p = case.payload[(r, i)].copy()
+                p[lo:hi].view("<u4")[0] ^= np.uint32(1)
+                tiers[r].put(case.keys[i], p, case.cks[(r, i)])
+            want = B.BSR_ERR_CHECKSUM
+        elif kind == "fill_error":
+            B.bsr_test_inject(gpu.ctx, B.BSR_INJECT_FILL_ERROR, r, 0, i, 0)
+            fetch_fault = lambda rr, ii: O.ERR_TRANSFER if (rr, ii) == (r, i) else None
+            want = B.BSR_ERR_TRANSFER
+        elif kind == "fill_stall":
+            B.bsr_test_inject(gpu.ctx, B.BSR_INJECT_FILL_STALL, r, 0, i, 0)
+            fetch_fault = lambda rr, ii: O.ERR_TIMEOUT if (rr, ii) == (r, i) else None
+            want = B.BSR_ERR_TIMEOUT
+        ora = _scrubbed_oracle(case, W, N, mutate_tiers=mutate, fetch_fault=fetch_fault)
+        assert ora["status"] == want
+        assert gpu.restore() == want
+        _check_failed(case, W, gpu, N, want, ora["paged"])
+        # the injected fault was one shot, tier corruption is not: a clean retry must succeed
+        if kind in ("corrupt_slot", "fill_error", "fill_stall"):
+            good = run_oracle(case, W)
+            gpu.B.bsr_reset_stats(gpu.ctx)
+            assert gpu.restore() == B.BSR_OK
+            _check_success(case, W, gpu, good, N)
+
+
+def test_commit_without_restore_and_after_invalidate():
+    case = Case(synth.tiny_layout(), 2, 6, seed=700)
+    ora = run_oracle(case, 2)
+    with GpuSide(case, 2) as gpu:
+        B = gpu.B
+        rc, keys, bm, n_hit = gpu.probe()
+        gpu.request(keys, n_hit)
+        assert gpu.commit() == 0                          # nothing restored yet
+        assert gpu.restore() == B.BSR_OK
+        assert gpu.commit() == 6 and gpu.commit() == 6    # idempotent
+        assert B.bsr_invalidate(gpu.ctx, gpu.req, 0) == B.BSR_OK
+        assert gpu.commit() == 0 and (gpu.bitmap(6) == 0).all()
+        assert_paged_equal(gpu, ora["paged"])             # invalidation without scrub moves no byte
+
+
+# ---------------------------------------------------------------- argument checking / edge cases
+def test_argument_errors_and_empty_request():
+    import torch
+    from paper_2608_17826_b200 import binding as B
+    assert B.bsr_ctx_create(0, 1)[0] == B.BSR_ERR_INVALID          # W = 0: legacy whole-plan mode
+    assert B.bsr_ctx_create(4, 0)[0] == B.BSR_ERR_INVALID
+    assert B.bsr_ctx_create(4, 9)[0] == B.BSR_ERR_INVALID
+    rc, ctx = B.bsr_ctx_create(4, 1)
+    assert rc == B.BSR_OK
+    buf = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda:0")
+    p = buf.data_ptr()
+    assert B.bsr_register(ctx, 0, [(64, 8)], [(0, 24, p)]) == B.BSR_ERR_ALIGN      # 24 % 16 != 0
+    assert B.bsr_register(ctx, 0, [(64, 8)], [(0, 32, p + 8)]) == B.BSR_ERR_ALIGN  # misaligned base
+    assert B.bsr_register(ctx, 0, [(48, 8)], [(0, 32, p)]) == B.BSR_ERR_INVALID    # 48 does not divide 256
+    assert B.bsr_register(ctx, 0, [(64, 8), (64, 8)], [(1, 32, p), (0, 32, p)]) == B.BSR_ERR_INVALID
+    assert B.bsr_register(ctx, 1, [(64, 8)], [(0, 32, p)]) == B.BSR_ERR_INVALID    # rank out of range
+    assert B.bsr_register(ctx, 0, [(64, 8)], [(0, 32, p)]) == B.BSR_OK
+    payload = np.zeros(256 * 32, dtype=np.uint8)
+    assert B.bsr_tier_put(ctx, 0, 1, payload, payload.size - 16, [0]) == B.BSR_ERR_INVALID
+    assert B.bsr_tier_put(ctx, 0, 1, payload, payload.size, [0]) == B.BSR_OK
+    keys = np.array([1], dtype=np.uint64)
+    assert B.bsr_req_create(ctx, keys, [np.array([0, 1, 2, 8], dtype=np.int32)])[0] == B.BSR_ERR_INVALID
+    assert B.bsr_req_create(ctx, keys, [np.array([0, 1, 2, 2], dtype=np.int32)])[0] == B.BSR_ERR_INVALID
+    assert B.bsr_req_create(ctx, keys, [np.array([0, 1, -1, 2], dtype=np.int32)])[0] == B.BSR_ERR_INVALID
+    assert "table" in B.bsr_last_error(ctx)
+    # an empty advertised prefix restores and commits to zero chunks
+    rc, req = B.bsr_req_create(ctx, keys[:0], [np.zeros(0, dtype=np.int32)])
+    assert rc == B.BSR_OK
+    assert B.bsr_restore(ctx, req) == B.BSR_OK
+    assert B.bsr_commit(ctx, req) == (B.BSR_OK, 0)
+    assert B.bsr_req_release(ctx, req) == B.BSR_OK
+    assert B.bsr_register(ctx, 0, [(64, 8)], [(0, 32, p)]) == B.BSR_ERR_STATE      # registration in use
+    assert B.bsr_ctx_destroy(ctx) == B.BSR_OK
