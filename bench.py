@@ -1,0 +1,390 @@
+#!/usr/bin/env python
+"""Benchmark of the bounded-state restore path on B200.
+
+One "step" is one pass of the whole hot path over one synthetic prefix: probe (chunk digests,
+key chain, index lookup) -> bounded-window restore (install kernels) -> commit.
+
+  value   restore throughput with the tier objects already resident in HBM (device tier): the
+          install kernels read them in place, no host link involved.
+  e2e     the same metric through the same C calls with the tier in ordinary HOST memory:
+          tier -> pinned W-slot ring -> cudaMemcpyAsync -> device staging -> install, every step.
+  roofline  the install kernel against the measured HBM copy bandwidth.
+  cpu_baseline  the CPU oracle timed on a bounded sample (reported, not a target).
+
+Usage: python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+Under torchrun (N > 1) every process drives its own GPU with its own copy of the workload
+(rank slices are independent units: weak scaling); the only exchange is the one-word commit AND.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2608_17826_b200 import synth  # noqa: E402
+
+WORKLOAD = dict(name="32768-token prefix, 128 chunks x 16,408,576 B, 2 rank slices, W=32, "
+                     "baseline 2-group/99-tensor layout, 64-token blocks",
+                n_chunks=128, n_ranks=2, W=32)
+METRIC, UNIT = "restore GB/s (all rank slices; per-rank = value / rank slices)", "GB/s"
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (earlier pool measurement)"
+
+
+class ClockSampler:
+    """Samples nvidia-smi SM clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        self.t.join(timeout=2)
+        sm = [float(r[0]) for r in self.rows if r and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) > 1 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for k, n in enumerate(names)
+                   if any(len(r) > 2 + k and r[2 + k].lower().startswith("active") for r in self.rows)]
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": reasons, "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------
+# CPU oracle legs (cpu_baseline of the default run, and --impl reference)
+# --------------------------------------------------------------------------------------------
+def oracle_sample_step(layout, n_ranks, sample_chunks, W, seed):
+    """One oracle pass (probe + strict-window restore + commit) over the first `sample_chunks`
+    chunks of the workload.  Returns (seconds, bytes moved)."""
+    from oracle import bsr_oracle as O
+    reg = O.Registration(list(layout.block_tokens), list(layout.tensors))
+    tok = synth.tokens(sample_chunks * 256, seed=seed)
+    keys = O.prefix_keys(O.chunk_digests(tok, seed), seed, 1)
+    tiers = [O.Tier() for _ in range(n_ranks)]
+    for r in range(n_ranks):
+        for i in range(sample_chunks):
+            p = synth.chunk_payload(layout, r, i, seed=seed).copy()
+            tiers[r].put(keys[i], p, O.group_checksums(reg, p))
+    pools = [synth.pool_blocks(layout, g, sample_chunks) for g in range(reg.n_groups)]
+    tables = [[synth.block_table(layout, r, g, sample_chunks, seed=seed) for g in range(reg.n_groups)]
+              for r in range(n_ranks)]
+    paged = [O.new_paged(reg, pools, synth.CANARY) for _ in range(n_ranks)]
+    t0 = time.perf_counter()
+    k, hit, n_hit = O.probe(tok, seed, 1, tiers)
+    req = O.Request(k[:n_hit], tables, n_ranks, reg.n_groups)
+    status, st = O.restore(reg, tiers, req, paged, W)
+    exposed = O.commit(reg, req, paged)
+    dt = time.perf_counter() - t0
+    assert status == O.OK and exposed == sample_chunks
+    return dt, n_ranks * sample_chunks * reg.chunk_bytes
+
+
+def run_reference(args):
+    """--impl reference: the oracle, as it stands, on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    layout = synth.baseline_layout()
+    sample = 8
+    for _ in range(args.warmup):
+        oracle_sample_step(layout, WORKLOAD["n_ranks"], sample, WORKLOAD["W"], synth.MASTER_SEED)
+    ts, nbytes = [], 0
+    for _ in range(args.steps):
+        dt, nbytes = oracle_sample_step(layout, WORKLOAD["n_ranks"], sample, WORKLOAD["W"], synth.MASTER_SEED)
+        ts.append(dt)
+    ms = 1e3 * sum(ts) / len(ts)
+    val = nbytes / (ms / 1e3) / 1e9
+    desc = f"first {sample} of {WORKLOAD['n_chunks']} chunks x {WORKLOAD['n_ranks']} rank slices per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u8/u64", "data": "synthetic",
+        "config": {"workload": WORKLOAD["name"], "sample": desc},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+    return 0
+
+
+# --------------------------------------------------------------------------------------------
+# GPU arm
+# --------------------------------------------------------------------------------------------
+class Side:
+    """A context with the workload registered and its tier filled, in host or device memory."""
+
+    def __init__(self, B, torch, dev, layout, n_ranks, n_chunks, W, payload_host, location, **cfg):
+        self.B, self.torch = B, torch
+        rc, self.ctx = B.bsr_ctx_create(W, n_ranks, device=dev.index, time_kernels=True, **cfg)
+        assert rc == B.BSR_OK, rc
+        self.G = layout.n_groups
+        pools = [synth.pool_blocks(layout, g, n_chunks) for g in range(self.G)]
+        self.paged = []
+        for r in range(n_ranks):
+            per = [torch.full((pools[g], layout.block_tokens[g], e), synth.CANARY, dtype=torch.uint8,
+                              device=dev) for g, e in layout.tensors]
+            self.paged.append(per)
+            rc = B.bsr_register(self.ctx, r, [(layout.block_tokens[g], pools[g]) for g in range(self.G)],
+                                [(g, e, per[l].data_ptr()) for l, (g, e) in enumerate(layout.tensors)])
+            assert rc == B.BSR_OK, B.bsr_last_error(self.ctx)
+        self.tables = [synth.block_table(layout, r, g, n_chunks) for r in range(n_ranks) for g in range(self.G)]
+        self.objs = payload_host if location == B.BSR_LOC_HOST else \
+            {k: torch.from_numpy(v).to(dev) for k, v in payload_host.items()}
+        self.location = location
+        self.req = None
+
+    def fill_tier(self, keys):
+        B = self.B
+        for (r, i), o in self.objs.items():
+            ptr = o if self.location == B.BSR_LOC_HOST else o.data_ptr()
+            n = o.size if self.location == B.BSR_LOC_HOST else o.numel()
+            rc = B.bsr_tier_put(self.ctx, r, keys[i], ptr, n, None, self.location)  # store path stamps checksums
+            assert rc == B.BSR_OK, B.bsr_last_error(self.ctx)
+
+    def step(self, tok, n_tok, salt, tok_on_device, stream):
+        B = self.B
+        rc, keys, bm, n_hit = B.bsr_probe(self.ctx, tok, n_tok, salt, tok_on_device)
+        assert rc == B.BSR_OK
+        if self.req is None:
+            rc, self.req = B.bsr_req_create(self.ctx, keys[:n_hit], self.tables)
+            assert rc == B.BSR_OK, B.bsr_last_error(self.ctx)
+        rc = B.bsr_restore(self.ctx, self.req, stream)
+        assert rc == B.BSR_OK, (rc, B.bsr_last_error(self.ctx))
+        rc, exposed = B.bsr_commit(self.ctx, self.req)
+        assert rc == B.BSR_OK
+        return n_hit, exposed
+
+    def stats(self):
+        return self.B.bsr_get_stats(self.ctx)[1]
+
+    def close(self):
+        if self.req is not None:
+            self.B.bsr_req_release(self.ctx, self.req)
+        self.B.bsr_ctx_destroy(self.ctx)
+
+
+def measure_h2d(torch, dev, piece_bytes, total_bytes=1 << 30, reps=5):
+    """Pinned-host -> device copy bandwidth in pieces of one chunk, best of reps (GB/s)."""
+    n = max(1, total_bytes // piece_bytes)
+    src = torch.empty(n * piece_bytes, dtype=torch.uint8).pin_memory()
+    dst = torch.empty(n * piece_bytes, dtype=torch.uint8, device=dev)
+    src.fill_(1)
+    best = 0.0
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for k in range(n):
+            dst[k * piece_bytes:(k + 1) * piece_bytes].copy_(src[k * piece_bytes:(k + 1) * piece_bytes],
+                                                            non_blocking=True)
+        e1.record()
+        torch.cuda.synchronize()
+        best = max(best, n * piece_bytes / (e0.elapsed_time(e1) / 1e3) / 1e9)
+    return best
+
+
+def timed_steps(torch, dist, world, side, tok, n_tok, salt, tok_on_device, steps, warmup, n_chunks):
+    stream = torch.cuda.current_stream()
+    for _ in range(warmup):
+        side.step(tok, n_tok, salt, tok_on_device, stream.cuda_stream)
+    side.B.bsr_reset_stats(side.ctx)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    ok = True
+    for _ in range(steps):
+        n_hit, exposed = side.step(tok, n_tok, salt, tok_on_device, stream.cuda_stream)
+        ok = ok and n_hit == n_chunks and exposed == n_chunks
+        if world > 1:  # request-level commit across GPUs: one word, AND over ranks (Eq. 6)
+            flag = torch.tensor([1 if exposed == n_chunks else 0], device="cuda", dtype=torch.int32)
+            dist.all_reduce(flag, op=dist.ReduceOp.MIN)
+            ok = ok and bool(flag.item())
+    e1.record(stream)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    assert ok, "a step did not expose the full prefix"
+    return ms / steps, side.stats()
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2608_17826_b200 import build
+    build.build()
+    from paper_2608_17826_b200 import binding as B  # raises if the CUDA library is missing
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the BSR path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    layout = synth.baseline_layout()
+    R, N, W = WORKLOAD["n_ranks"], args.chunks or WORKLOAD["n_chunks"], WORKLOAD["W"]
+    chunk = layout.chunk_bytes
+    seed = synth.MASTER_SEED + rank
+    salt = seed
+    tok = synth.tokens(N * 256, seed=seed)
+    payload = {(r, i): synth.chunk_payload(layout, r, i, seed=seed).copy() for r in range(R) for i in range(N)}
+    step_bytes = R * N * chunk
+
+    # ---- HBM-resident arm -----------------------------------------------------------------
+    d_tok = torch.from_numpy(tok).to(dev)
+    res = Side(B, torch, dev, layout, R, N, W, payload, B.BSR_LOC_DEVICE)
+    rc, keys, _, _ = B.bsr_probe(res.ctx, d_tok.data_ptr(), len(tok), salt, True)
+    assert rc == B.BSR_OK
+    res.fill_tier(keys)
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms_res, st_res = timed_steps(torch, dist, world, res, d_tok.data_ptr(), len(tok), salt, True,
+                                 args.steps, args.warmup, N)
+    launches = int(st_res.kernel_launches)
+    k_launches = int(st_res.install_launches)
+    k_ms = st_res.install_kernel_ms / max(1, k_launches)
+    res.close()
+    del res
+    torch.cuda.empty_cache()
+
+    if args.resident_only:  # profiling runs: only the HBM-resident arm, no JSON contract line
+        if rank == 0:
+            print(json.dumps({"resident_only": True, "chunks": N, "ms_per_step": ms_res,
+                              "install_launches": k_launches, "avg_launch_ms": k_ms,
+                              "GBps": step_bytes / (ms_res / 1e3) / 1e9}))
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    # ---- end-to-end arm: tier in host memory, through the pinned W-slot ring ----------------
+    h2d_gbs = measure_h2d(torch, dev, chunk)
+    e2e = Side(B, torch, dev, layout, R, N, W, payload, B.BSR_LOC_HOST,
+               load_concurrency=args.load_concurrency, dev_staging_depth=args.depth)
+    e2e.fill_tier(keys)
+    e2e_steps = max(3, min(args.steps, 10))
+    ms_e2e, st_e2e = timed_steps(torch, dist, world, e2e, tok, len(tok), salt, False, e2e_steps,
+                                 max(3, min(args.warmup, 3)), N)
+    peak_staging = [int(st_e2e.peak_staging_bytes[r]) for r in range(R)]
+    slot = int(st_e2e.slot_bytes)
+    clocks = sampler.stop()
+    e2e.close()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    hbm_peak, peak_src = _peaks()
+    value = world * step_bytes / (ms_res / 1e3) / 1e9
+    e2e_value = world * step_bytes / (ms_e2e / 1e3) / 1e9
+    per_launch_payload = step_bytes * args.steps / max(1, k_launches)
+    achieved = 2 * per_launch_payload / (k_ms / 1e3) / 1e9 if k_ms > 0 else None
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "install_traffic.json")
+    if os.path.exists(tpath):
+        with open(tpath) as f:
+            tj = json.load(f)
+        traffic = tj["dram_bytes_per_payload_byte"] * per_launch_payload
+
+    # ---- CPU oracle on a bounded sample -----------------------------------------------------
+    sample = 16
+    dt, nbytes = oracle_sample_step(layout, R, sample, W, seed)
+    cpu = {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+           "sample": f"first {sample} of {N} chunks x {R} rank slices, one pass ({dt:.1f} s)"}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_res, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u8 payload, u64 checksums/digests", "data": "synthetic",
+        "config": {"workload": WORKLOAD["name"] if N == WORKLOAD["n_chunks"] else f"REDUCED to {N} chunks: " + WORKLOAD["name"],
+                   "rank_slices_per_gpu": R, "W": W,
+                   "l2": "inputs (4.2 GB per step) are larger than L2; no flush needed",
+                   "value_path": "tier resident in HBM, probe+restore+commit",
+                   "e2e_path": f"host tier -> pinned ring -> H2D -> install; load_concurrency="
+                               f"{args.load_concurrency}, dev_staging_depth={args.depth}"},
+        "per_rank_GBps": value / (world * R),
+        "restore_seconds": ms_res / 1e3,
+        "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e, "steps": e2e_steps,
+                "h2d_bytes_per_step": step_bytes + len(tok) * 4,
+                "d2h_bytes_per_step": N * 8 + R * layout.n_groups * N * 12,
+                "per_rank_GBps": e2e_value / (world * R), "restore_seconds": ms_e2e / 1e3,
+                "h2d_link_GBps_measured": h2d_gbs, "frac_of_h2d_link": e2e_value / world / h2d_gbs},
+        "peak_staging_bytes_per_rank": peak_staging, "staging_law_bytes": W * slot,
+        "staging_residual_bytes": [p - W * slot for p in peak_staging],
+        "gpu_launches": launches,
+        "roofline": {"bound": "hbm", "kernel": "bsr_install_*_kernel", "achieved": achieved,
+                     "peak": hbm_peak, "unit": "GB/s", "frac": (achieved / hbm_peak) if achieved else None,
+                     "traffic": traffic, "peak_source": peak_src,
+                     "launches": k_launches, "avg_launch_ms": k_ms,
+                     "algorithmic_bytes_per_launch": 2 * per_launch_payload},
+        "cpu_baseline": cpu,
+        "clocks": clocks,
+    }
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--load-concurrency", type=int, default=8)
+    ap.add_argument("--depth", type=int, default=4)
+    ap.add_argument("--chunks", type=int, default=0, help="prefix length in chunks (default: the workload's 128)")
+    ap.add_argument("--resident-only", action="store_true", help="small profiling runs: skip e2e and CPU legs")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    return run_reference(args) if args.impl == "reference" else run_gpu(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())
