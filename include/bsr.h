@@ -245,6 +245,36 @@ enum {
 int bsr_test_inject(bsr_ctx *ctx, int kind, uint32_t rank, uint32_t group, uint32_t chunk,
                     uint64_t seed);
 
+/* ---- allocation-free prefix keys ----------------------------------------------------------- */
+
+#define BSR_NOALLOC_MAX_CHUNKS 8192u /* 2,097,152 tokens; the fixed scratch is 64 KiB + 256 B per GPU */
+
+/* The paper has no counterpart of this call; it exists for callers that cannot allocate.
+ *
+ * Who they are: an engine that has already given (nearly) all device memory to its KV block pool,
+ * where a cudaMalloc made later can simply fail; and scheduler-side code running between model
+ * steps, where the device-wide synchronisation hidden in cudaMalloc/cudaFree is not acceptable.
+ * bsr_probe grows its scratch with cudaMalloc on demand, so such callers use this instead.
+ *
+ * Computes the same prefix keys as bsr_probe (same digest, same chain, same reg_id mixing) for the
+ * n_tok / 256 full chunks of d_tok and writes them to d_keys_out, enqueued on `cuda_stream` (a
+ * cudaStream_t, NULL = the default stream).  It does not consult any index and returns as soon as
+ * the work is queued; the caller synchronises the stream before reading the keys.
+ *   d_tok       device, int32[n_tok], 16-byte aligned, caller-owned
+ *   d_keys_out  device, uint64[n_tok / 256], caller-owned
+ * The kernel's scratch lives in a fixed array inside the library image, so the call performs no
+ * cudaMalloc, cudaFree or other allocating routine.  Consequences the caller must know:
+ *   - at most BSR_NOALLOC_MAX_CHUNKS chunks per call; more is rejected with BSR_ERR_INVALID and a
+ *     message on stderr, nothing is launched;
+ *   - the first call on each GPU looks up the array's device address (one-time set-up); make that
+ *     first call outside any stream capture;
+ *   - all calls on one GPU share the one array: two calls whose kernels can overlap on the GPU
+ *     (different streams, no ordering between them) race and produce wrong keys.  Calls on one
+ *     stream, or otherwise ordered, are safe; each call clears what it needs before use.
+ * Errors: INVALID (device out of range, NULL pointer, too many chunks), ALIGN, CUDA. */
+int bsr_probe_keys_noalloc(int device, const int32_t *d_tok, size_t n_tok, uint64_t salt,
+                           uint64_t reg_id, uint64_t *d_keys_out, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

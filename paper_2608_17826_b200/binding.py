@@ -31,7 +31,9 @@ EXPORTS = [
     "bsr_tier_put", "bsr_tier_remove", "bsr_tier_checksums", "bsr_probe", "bsr_req_create",
     "bsr_req_release", "bsr_restore", "bsr_commit", "bsr_invalidate", "bsr_req_bitmap",
     "bsr_req_checksums", "bsr_get_stats", "bsr_reset_stats", "bsr_test_inject",
+    "bsr_probe_keys_noalloc",
 ]
+BSR_NOALLOC_MAX_CHUNKS = 8192
 
 
 class bsr_config(C.Structure):
@@ -87,6 +89,7 @@ def _load() -> C.CDLL:
         "bsr_get_stats": [vp, C.POINTER(bsr_stats)],
         "bsr_reset_stats": [vp],
         "bsr_test_inject": [vp, i32, u32, u32, u32, u64],
+        "bsr_probe_keys_noalloc": [i32, vp, C.c_size_t, u64, u64, vp, vp],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -221,3 +224,10 @@ def bsr_reset_stats(ctx) -> int:
 
 def bsr_test_inject(ctx, kind: int, rank: int = 0, group: int = 0, chunk: int = 0, seed: int = 0) -> int:
     return lib.bsr_test_inject(ctx, kind, rank, group, chunk, int(seed))
+
+
+def bsr_probe_keys_noalloc(device: int, d_tok: int, n_tok: int, salt: int, reg_id: int,
+                           d_keys_out: int, cuda_stream: int | None = None) -> int:
+    """Prefix keys for callers that must not allocate: device pointers in, device pointer out,
+    enqueued on `cuda_stream`; at most BSR_NOALLOC_MAX_CHUNKS chunks (see include/bsr.h)."""
+    return lib.bsr_probe_keys_noalloc(device, d_tok, n_tok, int(salt), int(reg_id), d_keys_out, cuda_stream)

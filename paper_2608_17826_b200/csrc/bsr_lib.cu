@@ -1106,3 +1106,88 @@ int bsr_test_inject(bsr_ctx *c, int kind, uint32_t rank, uint32_t group, uint32_
 }
 
 }  // extern "C"
+
+// =================================================================================================
+// Allocation-free prefix-key entry point
+// =================================================================================================
+// Some callers must not allocate.  A serving engine typically hands almost all of HBM to its KV
+// block pool at start-up, so a later cudaMalloc can fail outright; and cudaMalloc/cudaFree
+// synchronise the whole device, which a scheduler thread sitting between two model steps cannot
+// afford.  For them the probe kernel's scratch (the per-chunk digests and the block counter) lives
+// in a fixed array inside the library image instead of in memory obtained at run time.
+//
+// The array is part of the loaded module: every GPU that loads this library carries it
+// (BSR_NOALLOC_MAX_CHUNKS * 8 + 256 bytes) until the process exits.
+namespace {
+
+constexpr size_t kNoallocCounterWords = 32;  // 256 bytes reserved in front for the block counter
+static __device__ __align__(256) unsigned long long
+    bsr_noalloc_scratch[kNoallocCounterWords + BSR_NOALLOC_MAX_CHUNKS];
+
+constexpr int kNoallocMaxDevices = 64;
+std::mutex g_noalloc_mu;
+unsigned long long *g_noalloc_ptr[kNoallocMaxDevices] = {};  // device address of the array, per GPU
+
+}  // namespace
+
+extern "C" int bsr_probe_keys_noalloc(int device, const int32_t *d_tok, size_t n_tok, uint64_t salt,
+                                      uint64_t reg_id, uint64_t *d_keys_out, void *cuda_stream) {
+  const size_t N = n_tok / BSR_CHUNK_TOKENS;
+  if (device < 0 || device >= kNoallocMaxDevices) return BSR_ERR_INVALID;
+  if (N > BSR_NOALLOC_MAX_CHUNKS) {
+    fprintf(stderr,
+            "bsr_probe_keys_noalloc: %zu chunks exceed the fixed scratch of %u chunks "
+            "(BSR_NOALLOC_MAX_CHUNKS); use bsr_probe for longer prefixes\n",
+            N, (unsigned)BSR_NOALLOC_MAX_CHUNKS);
+    return BSR_ERR_INVALID;
+  }
+  if (N == 0) return BSR_OK;
+  if (!d_tok || !d_keys_out) return BSR_ERR_INVALID;
+  if ((reinterpret_cast<uintptr_t>(d_tok) & 15u) || (reinterpret_cast<uintptr_t>(d_keys_out) & 7u))
+    return BSR_ERR_ALIGN;
+  int prev = -1;
+  if (cudaGetDevice(&prev) != cudaSuccess) return BSR_ERR_CUDA;
+  if (prev != device && cudaSetDevice(device) != cudaSuccess) return BSR_ERR_CUDA;
+  int rc = BSR_OK;
+  unsigned long long *scratch = nullptr;
+  {
+    // Set-up, once per device, with that device current.  In host code the array's name is only a
+    // handle for the runtime; the address a kernel can use comes from cudaGetSymbolAddress.
+    std::lock_guard<std::mutex> lk(g_noalloc_mu);
+    if (!g_noalloc_ptr[device]) {
+      void *p = nullptr;
+      if (cudaGetSymbolAddress(&p, bsr_noalloc_scratch) != cudaSuccess || !p) {
+        cudaGetLastError();
+        rc = BSR_ERR_CUDA;
+      } else {
+        g_noalloc_ptr[device] = static_cast<unsigned long long *>(p);
+      }
+    }
+    scratch = g_noalloc_ptr[device];
+  }
+  if (rc == BSR_OK) {
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    unsigned int *counter = reinterpret_cast<unsigned int *>(scratch);
+    uint64_t *digests = reinterpret_cast<uint64_t *>(scratch + kNoallocCounterWords);
+    auto mix = [](uint64_t x) {
+      x += BSR_K_PHI;
+      x = (x ^ (x >> 32)) * BSR_K_PHI;
+      x = (x ^ (x >> 29)) * BSR_K_PHI;
+      return x ^ (x >> 32);
+    };
+    const uint64_t k_init = mix(salt ^ mix(reg_id));
+    const uint32_t per_block = BSR_K_PROBE_THREADS / 32;
+    const uint32_t grid = (uint32_t)((N + per_block - 1) / per_block);
+    // The array keeps whatever the previous call left.  Digests are fully rewritten for the N chunks
+    // that are read; the block counter must start at zero, so it is cleared in stream order.
+    if (cudaMemsetAsync(counter, 0, kNoallocCounterWords * 8, s) != cudaSuccess) {
+      rc = BSR_ERR_CUDA;
+    } else {
+      bsr_probe_kernel<<<grid, BSR_K_PROBE_THREADS, 0, s>>>(d_tok, (uint32_t)N, salt, k_init, digests,
+                                                            counter, d_keys_out);
+      if (cudaGetLastError() != cudaSuccess) rc = BSR_ERR_CUDA;
+    }
+  }
+  if (prev != device) cudaSetDevice(prev);
+  return rc;
+}
