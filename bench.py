@@ -376,7 +376,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
-    ap.add_argument("--load-concurrency", type=int, default=8)
+    ap.add_argument("--load-concurrency", type=int, default=0, help="fill threads (0 = auto)")
     ap.add_argument("--depth", type=int, default=4)
     ap.add_argument("--chunks", type=int, default=0, help="prefix length in chunks (default: the workload's 128)")
     ap.add_argument("--resident-only", action="store_true", help="small profiling runs: skip e2e and CPU legs")

@@ -3,6 +3,8 @@
 // The C interface is declared in include/bsr.h.
 #include "../../include/bsr.h"
 
+#include <immintrin.h>
+
 #include <atomic>
 #include <chrono>
 #include <condition_variable>
@@ -26,6 +28,7 @@ constexpr int kInstallThreads = 256;
 constexpr int kInstallUnroll = 4;
 constexpr int kLaunchSlots = 8;  // independent scratch sets for install launches in flight
 constexpr uint32_t kSmCount = 148;
+constexpr uint64_t kPieceBytes = 8ull << 20;  // fill and host-to-device copy granularity
 
 struct TierObj {
   const uint8_t *data;
@@ -121,6 +124,7 @@ struct bsr_ctx {
   std::vector<std::atomic<int>> *task_state = nullptr;  // 0 pending, 1 ready, <0 error
   std::vector<TierObj> *task_obj = nullptr;
   uint32_t fill_active = 0;
+  uint32_t pieces = 1;  // fill pieces per chunk
 
   Inject inject;
   bsr_stats st{};
@@ -233,9 +237,43 @@ int launch_install(bsr_ctx *c, const BsrInstallParams &p, cudaStream_t s) {
 }
 
 // ---- filler threads: tier object -> pinned slot -------------------------------------------------
+// Streaming copy for the fill: the destination slot will next be read by the copy engine, not by
+// this core, so non-temporal stores keep it out of the caches and spare the read-for-ownership.
+__attribute__((target("avx2"))) void stream_copy_avx2(uint8_t *dst, const uint8_t *src, size_t n) {
+  size_t i = 0;
+  while (i < n && (reinterpret_cast<uintptr_t>(dst + i) & 31u)) {
+    dst[i] = src[i];
+    ++i;
+  }
+  for (; i + 128 <= n; i += 128) {
+    _mm_prefetch(reinterpret_cast<const char *>(src + i + 1024), _MM_HINT_NTA);
+    const __m256i a = _mm256_loadu_si256(reinterpret_cast<const __m256i *>(src + i));
+    const __m256i b = _mm256_loadu_si256(reinterpret_cast<const __m256i *>(src + i + 32));
+    const __m256i c2 = _mm256_loadu_si256(reinterpret_cast<const __m256i *>(src + i + 64));
+    const __m256i d = _mm256_loadu_si256(reinterpret_cast<const __m256i *>(src + i + 96));
+    _mm256_stream_si256(reinterpret_cast<__m256i *>(dst + i), a);
+    _mm256_stream_si256(reinterpret_cast<__m256i *>(dst + i + 32), b);
+    _mm256_stream_si256(reinterpret_cast<__m256i *>(dst + i + 64), c2);
+    _mm256_stream_si256(reinterpret_cast<__m256i *>(dst + i + 96), d);
+  }
+  _mm_sfence();
+  for (; i < n; ++i) dst[i] = src[i];
+}
+
+void fill_copy(uint8_t *dst, const uint8_t *src, size_t n) {
+  static const bool avx2 = __builtin_cpu_supports("avx2");
+  if (avx2 && n >= 4096)
+    stream_copy_avx2(dst, src, n);
+  else
+    memcpy(dst, src, n);
+}
+
+// One fill task = one piece (at most kPieceBytes) of one chunk of one rank.  Pieces let the first
+// device copy start after a fraction of a chunk has been fetched and keep all threads busy on the
+// chunks the copy engine needs next.
 void filler_main(bsr_ctx *c) {
   for (;;) {
-    uint32_t s;
+    uint32_t t;
     bsr_req *req;
     {
       std::unique_lock<std::mutex> lk(c->fill_mu);
@@ -243,12 +281,15 @@ void filler_main(bsr_ctx *c) {
         return c->fill_shutdown || (c->cur_req && c->fill_next < c->fill_admitted);
       });
       if (c->fill_shutdown) return;
-      s = c->fill_next++;
+      t = c->fill_next++;
       req = c->cur_req;
       c->fill_active++;
     }
-    const uint32_t R = c->cfg.n_ranks, W = c->cfg.window_chunks;
+    const uint32_t R = c->cfg.n_ranks, W = c->cfg.window_chunks, P = c->pieces;
+    const uint32_t s = t / P, piece = t % P;
     const uint32_t i = s / R, r = s % R;
+    const uint64_t off = (uint64_t)piece * kPieceBytes;
+    const uint64_t len = (c->chunk_bytes - off < kPieceBytes) ? c->chunk_bytes - off : kPieceBytes;
     int state = 1;
     TierObj obj{};
     if (!c->fill_abort.load(std::memory_order_acquire)) {
@@ -267,23 +308,24 @@ void filler_main(bsr_ctx *c) {
         state = BSR_ERR_MISSING;
       } else if (hit && inj.kind == BSR_INJECT_FILL_ERROR) {
         state = BSR_ERR_TRANSFER;
-      } else if (hit && inj.kind == BSR_INJECT_FILL_STALL) {
+      } else if (hit && inj.kind == BSR_INJECT_FILL_STALL && piece == 0) {
         while (!c->fill_abort.load(std::memory_order_acquire) &&
                Clock::now() < c->fill_deadline + std::chrono::seconds(5))
           std::this_thread::sleep_for(std::chrono::milliseconds(1));
         state = BSR_ERR_TIMEOUT;
       } else if (obj.loc == BSR_LOC_HOST) {
         uint8_t *slot = c->ring[r] + (size_t)(i % W) * c->slot_bytes;
-        memcpy(slot, obj.data, obj.len);
+        fill_copy(slot + off, obj.data + off, len);
         if (hit && inj.kind == BSR_INJECT_CORRUPT_SLOT && inj.group < c->G) {
           const uint64_t words = c->seg_bytes[inj.group] / 4;
-          uint32_t *w = reinterpret_cast<uint32_t *>(slot + c->seg_begin[inj.group]);
-          w[inj.seed % words] ^= (uint32_t)(0x80000000u >> (inj.seed % 31));
+          const uint64_t at = c->seg_begin[inj.group] + 4 * (inj.seed % words);
+          if (at >= off && at < off + len)
+            *reinterpret_cast<uint32_t *>(slot + at) ^= (uint32_t)(0x80000000u >> (inj.seed % 31));
         }
       }
     }
-    (*c->task_obj)[s] = obj;
-    (*c->task_state)[s].store(state, std::memory_order_release);
+    if (piece == 0) (*c->task_obj)[s] = obj;
+    (*c->task_state)[t].store(state, std::memory_order_release);
     {
       std::lock_guard<std::mutex> lk(c->fill_mu);
       c->fill_active--;
@@ -429,13 +471,14 @@ int restore_ring(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_point 
   if (rc != BSR_OK) return rc;
   const uint32_t R = c->cfg.n_ranks, W = c->cfg.window_chunks, D = c->cfg.dev_staging_depth;
   const uint32_t N = q->n_adv, total = N * R;
-  std::vector<std::atomic<int>> state(total);
+  const uint32_t P = c->pieces;
+  std::vector<std::atomic<int>> state((size_t)total * P);  // per piece: 0 pending, 1 ready, <0 error
   for (auto &s : state) s.store(0, std::memory_order_relaxed);
   std::vector<TierObj> objs(total);
   {
     std::lock_guard<std::mutex> lk(c->fill_mu);
     c->cur_req = q;
-    c->fill_total = total;
+    c->fill_total = total * P;
     c->fill_admitted = 0;
     c->fill_next = 0;
     c->fill_abort.store(false);
@@ -443,7 +486,7 @@ int restore_ring(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_point 
     c->task_state = &state;
     c->task_obj = &objs;
   }
-  uint32_t admitted = 0, submitted = 0, reaped = 0;
+  uint32_t admitted = 0, submitted = 0, reaped = 0, cur_piece = 0;
   uint32_t released[BSR_MAX_RANKS] = {};
   for (uint32_t r = 0; r < R; ++r) c->live[r] = 0;
   bool stop = false;  // a failure was seen: admit and submit nothing more, drain
@@ -472,7 +515,7 @@ int restore_ring(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_point 
       if (n_new) {
         {
           std::lock_guard<std::mutex> lk(c->fill_mu);
-          c->fill_admitted = admitted;
+          c->fill_admitted = admitted * P;
         }
         c->fill_cv.notify_all();
         progress = true;
@@ -500,32 +543,51 @@ int restore_ring(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_point 
       ++reaped;
       progress = true;
     }
-    // submit, in order: slot -> device staging on the copy stream, then the install kernel
+    // submit, in order: every ready piece slot -> device staging on the copy stream; when the chunk
+    // is complete, the install kernel on the compute stream
     while (!stop && submitted < admitted && submitted - reaped < R * D) {
-      const int stt = state[submitted].load(std::memory_order_acquire);
-      if (stt == 0) break;
-      if (stt < 0) {
-        first_error(stt);
-        break;
-      }
       const uint32_t i = submitted / R, r = submitted % R, d = i % D, k = r * D + d;
-      const TierObj &o = objs[submitted];
       uint8_t *stage = c->dstage[r] + (size_t)d * c->chunk_bytes;
-      const uint8_t *from = (o.loc == BSR_LOC_HOST) ? c->ring[r] + (size_t)(i % W) * c->slot_bytes
-                                                    : o.data;
-      cudaError_t e = cudaStreamWaitEvent(c->copy_stream, c->ev_inst[k], 0);
-      if (e == cudaSuccess)
-        e = cudaMemcpyAsync(stage, from, c->chunk_bytes, cudaMemcpyDefault, c->copy_stream);
-      if (e == cudaSuccess) e = cudaEventRecord(c->ev_h2d[k], c->copy_stream);
+      cudaError_t e = cudaSuccess;
+      bool blocked = false;
+      while (cur_piece < P) {
+        const int stt = state[(size_t)submitted * P + cur_piece].load(std::memory_order_acquire);
+        if (stt == 0) {
+          blocked = true;
+          break;
+        }
+        if (stt < 0) {
+          first_error(stt);
+          break;
+        }
+        const TierObj &o = objs[submitted];
+        const uint64_t off = (uint64_t)cur_piece * kPieceBytes;
+        const uint64_t len = (c->chunk_bytes - off < kPieceBytes) ? c->chunk_bytes - off : kPieceBytes;
+        const uint8_t *from = (o.loc == BSR_LOC_HOST)
+                                  ? c->ring[r] + (size_t)(i % W) * c->slot_bytes + off
+                                  : o.data + off;
+        if (cur_piece == 0) e = cudaStreamWaitEvent(c->copy_stream, c->ev_inst[k], 0);
+        if (e == cudaSuccess)
+          e = cudaMemcpyAsync(stage + off, from, len, cudaMemcpyDefault, c->copy_stream);
+        if (e != cudaSuccess) {
+          first_error(fail(c, BSR_ERR_TRANSFER, "copy submit: %s", cudaGetErrorString(e)));
+          break;
+        }
+        c->st.h2d_copies++;
+        c->st.bytes_filled[r] += (o.loc == BSR_LOC_HOST) ? len : 0;
+        c->st.bytes_h2d[r] += len;
+        ++cur_piece;
+        progress = true;
+      }
+      if (stop || blocked) break;
+      const TierObj &o = objs[submitted];
+      e = cudaEventRecord(c->ev_h2d[k], c->copy_stream);
       if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, c->ev_h2d[k], 0);
       if (e == cudaSuccess && c->cfg.time_kernels) e = cudaEventRecord(c->ev_start[k], stream);
       if (e != cudaSuccess) {
         first_error(fail(c, BSR_ERR_TRANSFER, "copy submit: %s", cudaGetErrorString(e)));
         break;
       }
-      c->st.h2d_copies++;
-      c->st.bytes_filled[r] += (o.loc == BSR_LOC_HOST) ? c->chunk_bytes : 0;
-      c->st.bytes_h2d[r] += c->chunk_bytes;
       BsrInstallParams p{};
       fill_params(c, p, (uint32_t)(c->launch_seq++ % kLaunchSlots));
       p.n_adv = N;
@@ -545,6 +607,7 @@ int restore_ring(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_point 
         break;
       }
       ++submitted;
+      cur_piece = 0;
       progress = true;
     }
     if (reaped == submitted && (stop || reaped == total)) break;
@@ -559,6 +622,8 @@ int restore_ring(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_point 
       std::this_thread::yield();
     }
   }
+  // copies of a chunk that never reached its install launch may still be queued
+  if (cur_piece != 0) cudaStreamSynchronize(c->copy_stream);
   // quiesce the fillers: nothing of this request may be touched after return
   c->fill_abort.store(true, std::memory_order_release);
   {
@@ -593,7 +658,10 @@ int bsr_ctx_create(const bsr_config *cfg, bsr_ctx **out) {
   bsr_ctx *c = new (std::nothrow) bsr_ctx();
   if (!c) return BSR_ERR_NOMEM;
   c->cfg = *cfg;
-  if (c->cfg.load_concurrency == 0) c->cfg.load_concurrency = 4;
+  if (c->cfg.load_concurrency == 0) {  // auto: one copy thread per two hardware threads, 4..16
+    const unsigned hw = std::thread::hardware_concurrency() / 2;
+    c->cfg.load_concurrency = hw < 4 ? 4 : (hw > 16 ? 16 : hw);
+  }
   if (c->cfg.load_concurrency > 64) c->cfg.load_concurrency = 64;
   if (c->cfg.dev_staging_depth == 0) c->cfg.dev_staging_depth = 4;
   if (c->cfg.dev_staging_depth > 16) c->cfg.dev_staging_depth = 16;
@@ -707,6 +775,7 @@ int bsr_register(bsr_ctx *c, uint32_t rank, const bsr_group_desc *groups, uint32
       off += sz;
     }
     c->chunk_bytes = off;
+    c->pieces = (uint32_t)((off + kPieceBytes - 1) / kPieceBytes);
     c->slot_bytes = round_up(off, c->cfg.slot_align);
     c->st.slot_bytes = c->slot_bytes;
   } else {
