@@ -239,19 +239,25 @@ class Stats:
 # --------------------------------------------------------------------------------------
 # install  (Section 2 "Bounded installation", Section 3 "Install locally")
 # --------------------------------------------------------------------------------------
+def block_of_chunk(reg: Registration, chunk: np.ndarray, l: int, b: int) -> np.ndarray:
+    """The rows [B_g, e_l] that a chunk carries for tensor l and the chunk's logical block b:
+    tokens b*B_g .. (b+1)*B_g - 1 of the tensor's [256, e_l] slab at byte offset tensor_offset(l)."""
+    g, e = reg.tensors[l]
+    B = reg.block_tokens[g]
+    off = reg.tensor_offset(l) + b * B * e
+    return chunk[off: off + B * e].reshape(B, e)
+
+
 def scatter_chunk_group(reg: Registration, g: int, chunk: np.ndarray, i: int,
                         table: np.ndarray, paged: list[np.ndarray]):
     """Install group g of chunk i: token t of the chunk (global token 256 i + t) of tensor l goes
     to paged[l][ table[(256 i + t) // B_g], (256 i + t) % B_g, : ]."""
-    B = reg.block_tokens[g]
     nb = reg.blocks_per_chunk(g)
-    for l, (gg, e) in enumerate(reg.tensors):
+    for l, (gg, _) in enumerate(reg.tensors):
         if gg != g:
             continue
-        off = reg.tensor_offset(l)
-        src = chunk[off: off + CHUNK_TOKENS * e].reshape(nb, B, e)
         for b in range(nb):
-            paged[l][table[i * nb + b]] = src[b]
+            paged[l][table[i * nb + b]] = block_of_chunk(reg, chunk, l, b)
 
 
 def restore(reg: Registration, tiers: list[Tier], req: Request, paged: list[list[np.ndarray]],

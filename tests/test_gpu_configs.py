@@ -1,0 +1,248 @@
+"""The five workload configurations at their full sizes on a B200, against the oracle.
+
+Configuration 2 (the benchmarked one) is fully materialised and every paged byte is compared,
+in both launch configurations the benchmark times (device-resident tier: 64 chunk descriptors
+per install launch; host tier: ring + one chunk per launch).  Configurations 3-5 move 8-67 GB
+per rank; there the host tier is cyclic (P distinct seeded objects per rank, P prime and > W,
+key i -> object i mod P) so that the oracle can checksum every object, and the result is checked
+through: every (rank, group, chunk) checksum the install kernel computed == the oracle's checksum
+of the object that chunk maps to; sampled destination blocks == the oracle's block of that object;
+spare blocks still hold the canary; bitmap, exposure, windows, byte counters and the staging law.
+"""
+import numpy as np
+import pytest
+
+from conftest import read_golden
+from harness import Case, GpuSide, assert_paged_equal, run_oracle
+from oracle import bsr_oracle as O
+from paper_2608_17826_b200 import synth
+
+pytestmark = pytest.mark.gpu
+COEFF = int(read_golden("paper_capacity.txt")["law_coefficient"])
+
+
+# ---------------------------------------------------------------- configuration 2, every byte
+def test_config2_every_paged_byte_both_launch_configurations():
+    layout = synth.baseline_layout()
+    R, N, W = 2, 128, 32
+    case = Case(layout, R, N, seed=synth.MASTER_SEED)
+    ora = run_oracle(case, W)
+    assert ora["status"] == O.OK and ora["exposed"] == N
+    assert ora["stats"].peak_staging_bytes == [W * COEFF] * R
+    for location in (0, 1):
+        with GpuSide(case, W, location=location) as gpu:
+            B = gpu.B
+            rc, keys, bm, n_hit = gpu.probe()
+            assert rc == B.BSR_OK and n_hit == N and np.array_equal(keys, ora["keys"])
+            gpu.request(keys, N)
+            assert gpu.restore() == B.BSR_OK, B.bsr_last_error(gpu.ctx)
+            assert gpu.commit() == N
+            assert np.array_equal(gpu.bitmap(N), ora["req"].bitmap())
+            st = gpu.stats()
+            for r in range(R):
+                assert st.bytes_installed[r] == N * COEFF == 2_100_297_728
+                if location == 0:
+                    assert st.peak_staging_bytes[r] == 32 * COEFF == 525_074_432   # Eq. 5, residual 0
+                    assert st.bytes_filled[r] == st.bytes_h2d[r] == N * COEFF
+            assert st.windows == 4
+            assert_paged_equal(gpu, ora["paged"])
+
+
+# ---------------------------------------------------------------- big cases with a cyclic tier
+_OBJ_CACHE: dict = {}
+
+
+class CyclicCase:
+    def __init__(self, layout, R, N, P, seed, present=None):
+        self.layout, self.R, self.N, self.P, self.seed = layout, R, N, P, seed
+        self.reg = O.Registration(list(layout.block_tokens), list(layout.tensors))
+        self.G = self.reg.n_groups
+        self.tok = synth.tokens(N * 256, seed=seed)
+        self.salt = seed
+        self.keys = O.prefix_keys(O.chunk_digests(self.tok, self.salt), self.salt, 1)
+        ck = (layout.name, R, P)          # payload objects depend on the layout only: build them once
+        if ck not in _OBJ_CACHE:
+            objs = {(r, j): synth.chunk_payload(layout, r, j, seed=synth.MASTER_SEED + 1).copy()
+                    for r in range(R) for j in range(P)}
+            _OBJ_CACHE[ck] = (objs, {k: O.group_checksums(self.reg, v) for k, v in objs.items()})
+        self.objs, self.cks = _OBJ_CACHE[ck]
+        self.present = present or (lambda r, i: True)
+        self.pools = [synth.pool_blocks(layout, g, N) for g in range(self.G)]
+        self.tables = [[synth.block_table(layout, r, g, N, seed=seed) for g in range(self.G)]
+                       for r in range(R)]
+
+
+class BigGpu:
+    def __init__(self, case: CyclicCase, W, **cfg):
+        import torch
+        from paper_2608_17826_b200 import binding as B
+        self.B, self.torch, self.case = B, torch, case
+        dev = torch.device("cuda:0")
+        rc, self.ctx = B.bsr_ctx_create(W, case.R, **cfg)
+        assert rc == B.BSR_OK
+        self.paged = []
+        for r in range(case.R):
+            per = [torch.full((case.pools[g], case.layout.block_tokens[g], e), synth.CANARY,
+                              dtype=torch.uint8, device=dev) for g, e in case.layout.tensors]
+            self.paged.append(per)
+            rc = B.bsr_register(self.ctx, r, [(case.layout.block_tokens[g], case.pools[g]) for g in range(case.G)],
+                                [(g, e, per[l].data_ptr()) for l, (g, e) in enumerate(case.layout.tensors)])
+            assert rc == B.BSR_OK, B.bsr_last_error(self.ctx)
+        for r in range(case.R):
+            for i in range(case.N):
+                if case.present(r, i):
+                    o = case.objs[(r, i % case.P)]
+                    assert B.bsr_tier_put(self.ctx, r, case.keys[i], o, o.size, case.cks[(r, i % case.P)]) == B.BSR_OK
+        self.req = None
+
+    def request(self, n_adv):
+        c = self.case
+        flat = [c.tables[r][g][: n_adv * c.reg.blocks_per_chunk(g)] for r in range(c.R) for g in range(c.G)]
+        rc, self.req = self.B.bsr_req_create(self.ctx, c.keys[:n_adv], flat)
+        assert rc == self.B.BSR_OK, self.B.bsr_last_error(self.ctx)
+
+    def check_success(self, W, n_adv, samples=1500):
+        B, c, torch = self.B, self.case, self.torch
+        assert B.bsr_commit(self.ctx, self.req) == (B.BSR_OK, n_adv)
+        rc, bm = B.bsr_req_bitmap(self.ctx, self.req, c.R, c.G, n_adv)
+        want_row = O.pack_bits(np.ones(n_adv, dtype=bool))
+        assert np.array_equal(bm, np.tile(want_row, c.R * c.G))
+        st = B.bsr_get_stats(self.ctx)[1]
+        assert st.windows == -(-n_adv // W)                                   # K = ceil(N / W)
+        for r in range(c.R):
+            assert st.peak_staging_bytes[r] == min(W, n_adv) * c.reg.slot_bytes     # Eq. 5
+            assert st.bytes_filled[r] == st.bytes_h2d[r] == st.bytes_installed[r] == n_adv * c.reg.chunk_bytes
+        # every checksum the kernel computed, against the oracle's checksum of the mapped object
+        rc, cks = B.bsr_req_checksums(self.ctx, self.req, c.R, c.G, n_adv)
+        for r in range(c.R):
+            want = np.array([c.cks[(r, i % c.P)] for i in range(n_adv)], dtype=np.uint64).T
+            assert np.array_equal(cks[r], want)
+        # sampled destination blocks against the oracle's block of the mapped object
+        rng = np.random.default_rng(c.seed)
+        for _ in range(samples):
+            r = int(rng.integers(0, c.R))
+            l = int(rng.integers(0, len(c.layout.tensors)))
+            g = c.layout.tensors[l][0]
+            nb = c.reg.blocks_per_chunk(g)
+            j = int(rng.integers(0, n_adv * nb))
+            want = O.block_of_chunk(c.reg, c.objs[(r, (j // nb) % c.P)], l, j % nb)
+            got = self.paged[r][l][int(c.tables[r][g][j])].cpu().numpy()
+            assert np.array_equal(got, want), (r, l, j)
+        self.check_untouched(n_adv)
+
+    def check_untouched(self, n_adv):
+        """Blocks outside the request's tables still hold the canary."""
+        c, torch = self.case, self.torch
+        for r in range(c.R):
+            for g in range(c.G):
+                used = np.zeros(c.pools[g], dtype=bool)
+                used[c.tables[r][g][: n_adv * c.reg.blocks_per_chunk(g)]] = True
+                spare = torch.from_numpy(np.flatnonzero(~used)).cuda()
+                for l, (gg, _) in enumerate(c.layout.tensors):
+                    if gg == g:
+                        assert bool((self.paged[r][l][spare] == synth.CANARY).all())
+
+    def check_scrubbed(self, n_adv):
+        c, torch = self.case, self.torch
+        for r in range(c.R):
+            for g in range(c.G):
+                used = torch.from_numpy(c.tables[r][g][: n_adv * c.reg.blocks_per_chunk(g)].astype(np.int64)).cuda()
+                for l, (gg, _) in enumerate(c.layout.tensors):
+                    if gg == g:
+                        assert bool((self.paged[r][l][used] == 0).all())
+        self.check_untouched(n_adv)
+
+    def close(self):
+        if self.req is not None:
+            self.B.bsr_req_release(self.ctx, self.req)
+        self.B.bsr_ctx_destroy(self.ctx)
+        self.paged = None
+        self.torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("N", [512, 1024])
+def test_config3_window_sweep_staging_law(N):
+    layout = synth.baseline_layout()
+    case = CyclicCase(layout, 2, N, P=67, seed=3003 + N)
+    g = read_golden("paper_capacity.txt")
+    for W in (8, 16, 32, 64):
+        gpu = BigGpu(case, W)
+        try:
+            rc, keys, bm, n_hit = gpu.B.bsr_probe(gpu.ctx, case.tok, len(case.tok), case.salt)
+            assert rc == gpu.B.BSR_OK and n_hit == N and np.array_equal(keys, case.keys)
+            gpu.request(N)
+            assert gpu.B.bsr_restore(gpu.ctx, gpu.req) == gpu.B.BSR_OK, gpu.B.bsr_last_error(gpu.ctx)
+            gpu.check_success(W, N, samples=400)
+            st = gpu.B.bsr_get_stats(gpu.ctx)[1]
+            assert st.peak_staging_bytes[0] == st.peak_staging_bytes[1] == float(g[f"rws_mib_w{W}"]) * 2**20
+        finally:
+            gpu.close()
+
+
+@pytest.mark.parametrize("layout_name", ["baseline", "hetero"])
+def test_config4_2048_chunks(layout_name):
+    layout = synth.baseline_layout() if layout_name == "baseline" else synth.hetero_layout()
+    N, W = 2048, 32
+    case = CyclicCase(layout, 2, N, P=67, seed=4004)
+    gpu = BigGpu(case, W)
+    try:
+        rc, keys, bm, n_hit = gpu.B.bsr_probe(gpu.ctx, case.tok, len(case.tok), case.salt)
+        assert rc == gpu.B.BSR_OK and n_hit == N and np.array_equal(keys, case.keys)
+        gpu.request(N)
+        assert gpu.B.bsr_restore(gpu.ctx, gpu.req) == gpu.B.BSR_OK, gpu.B.bsr_last_error(gpu.ctx)
+        gpu.check_success(W, N)
+        st = gpu.B.bsr_get_stats(gpu.ctx)[1]
+        assert st.bytes_installed[0] == 33_604_763_648 and st.peak_staging_bytes[0] == 525_074_432
+    finally:
+        gpu.close()
+
+
+@pytest.mark.parametrize("kind", ["checksum", "missing", "rank_asymmetric", "partial_hit"])
+def test_config5_failures_at_1024_chunks(kind):
+    layout = synth.baseline_layout()
+    R, N, W = 2, 1024, 16
+    present = (lambda r, i: i < 700 or i == 800) if kind == "partial_hit" else None
+    case = CyclicCase(layout, R, N, P=67, seed=5005, present=present)
+    gpu = BigGpu(case, W)
+    B = gpu.B
+    try:
+        rc, keys, bm, n_hit = B.bsr_probe(gpu.ctx, case.tok, len(case.tok), case.salt)
+        assert rc == B.BSR_OK and np.array_equal(keys, case.keys)
+        if kind == "partial_hit":
+            hit = np.array([i < 700 or i == 800 for i in range(N)])
+            assert n_hit == 700 and np.array_equal(bm, O.pack_bits(hit))
+            gpu.request(700)
+            assert B.bsr_restore(gpu.ctx, gpu.req) == B.BSR_OK
+            gpu.check_success(W, 700, samples=400)
+            st = B.bsr_get_stats(gpu.ctx)[1]
+            assert st.windows == 44 and st.bytes_installed[0] == 11_486_003_200
+            return
+        assert n_hit == N
+        gpu.request(N)
+        r, g, i, frac = synth.fault_site(R, case.G, W, N, case={"checksum": 0, "missing": 1, "rank_asymmetric": 2}[kind])
+        if kind == "rank_asymmetric":
+            r, g = 1, 1
+        if kind == "missing":
+            assert B.bsr_tier_remove(gpu.ctx, r, case.keys[i]) == B.BSR_OK
+            want = B.BSR_ERR_MISSING
+        else:
+            # the cyclic tier shares objects between chunks: give chunk i a private corrupted copy
+            bad = case.objs[(r, i % case.P)].copy()
+            lo, hi = case.reg.segment(g)
+            w = bad[lo:hi].view("<u4")
+            w[frac % len(w)] ^= np.uint32(1 << (frac % 32))
+            assert B.bsr_tier_put(gpu.ctx, r, case.keys[i], bad, bad.size, case.cks[(r, i % case.P)]) == B.BSR_OK
+            want = B.BSR_ERR_CHECKSUM
+        assert B.bsr_restore(gpu.ctx, gpu.req) == want
+        assert B.bsr_commit(gpu.ctx, gpu.req) == (B.BSR_OK, 0)
+        rc, bmv = B.bsr_req_bitmap(gpu.ctx, gpu.req, R, case.G, N)
+        assert (bmv == 0).all()                                   # the healthy rank's bits too
+        st = B.bsr_get_stats(gpu.ctx)[1]
+        assert 0 < max(st.peak_staging_bytes[:R]) <= W * COEFF
+        assert max(st.bytes_installed[:R]) < N * COEFF            # stopped early
+        gpu.check_untouched(N)
+        assert B.bsr_invalidate(gpu.ctx, gpu.req, B.BSR_SCRUB) == B.BSR_OK
+        gpu.check_scrubbed(N)
+        assert B.bsr_commit(gpu.ctx, gpu.req) == (B.BSR_OK, 0)
+    finally:
+        gpu.close()
