@@ -276,7 +276,7 @@ def run_gpu(args):
 
     # ---- HBM-resident arm -----------------------------------------------------------------
     d_tok = torch.from_numpy(tok).to(dev)
-    res = Side(B, torch, dev, layout, R, N, W, payload, B.BSR_LOC_DEVICE)
+    res = Side(B, torch, dev, layout, R, N, W, payload, B.BSR_LOC_DEVICE, install_variant=args.variant)
     rc, keys, _, _ = B.bsr_probe(res.ctx, d_tok.data_ptr(), len(tok), salt, True)
     assert rc == B.BSR_OK
     res.fill_tier(keys)
@@ -303,7 +303,8 @@ def run_gpu(args):
     # ---- end-to-end arm: tier in host memory, through the pinned W-slot ring ----------------
     h2d_gbs = measure_h2d(torch, dev, chunk)
     e2e = Side(B, torch, dev, layout, R, N, W, payload, B.BSR_LOC_HOST,
-               load_concurrency=args.load_concurrency, dev_staging_depth=args.depth)
+               load_concurrency=args.load_concurrency, dev_staging_depth=args.depth,
+               install_variant=args.variant)
     e2e.fill_tier(keys)
     e2e_steps = max(3, min(args.steps, 10))
     ms_e2e, st_e2e = timed_steps(torch, dist, world, e2e, tok, len(tok), salt, False, e2e_steps,
@@ -378,6 +379,7 @@ def main():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--load-concurrency", type=int, default=0, help="fill threads (0 = auto)")
     ap.add_argument("--depth", type=int, default=4)
+    ap.add_argument("--variant", type=int, default=0, help="install kernel: 0 auto, 1 vector, 2 bulk copy")
     ap.add_argument("--chunks", type=int, default=0, help="prefix length in chunks (default: the workload's 128)")
     ap.add_argument("--resident-only", action="store_true", help="small profiling runs: skip e2e and CPU legs")
     args = ap.parse_args()

@@ -54,8 +54,13 @@ struct BsrInstallParams {
   unsigned int *err_flag;    // set to nonzero if a bounded wait gave up (bulk variant)
   uint64_t *ck_out;          // [(r*G + g) * n_adv + i] computed checksum
   uint32_t *verdict;         // same index: 1 verified, 2 mismatch
-  BsrChunkDesc chunk[BSR_K_MAX_BATCH];
+  const BsrChunkDesc *batch; // device array of n_chunks descriptors, or NULL: use `one`
+  BsrChunkDesc one;          // the descriptor of a single-chunk launch, carried in the parameters
 };
+
+__device__ __forceinline__ const BsrChunkDesc *bsr_desc(const BsrInstallParams &p, uint32_t c) {
+  return p.batch ? p.batch + c : &p.one;
+}
 
 // ---------------------------------------------------------------------------------------------
 // helpers
@@ -134,7 +139,7 @@ __device__ __forceinline__ void bsr_install_finish(const BsrInstallParams &p) {
     uint64_t *a = p.acc + c * BSR_K_MAX_GROUPS + g;
     const uint64_t s = __ldcg((const unsigned long long *)a);
     *a = 0ull;
-    const BsrChunkDesc &cd = p.chunk[c];
+    const BsrChunkDesc &cd = *bsr_desc(p, c);
     const size_t o = ((size_t)cd.rank * G + g) * p.n_adv + cd.chunk;
     p.ck_out[o] = s;
     p.verdict[o] = (s == cd.expect[g]) ? 1u : 2u;
@@ -165,7 +170,7 @@ bsr_install_vec_kernel(const __grid_constant__ BsrInstallParams p) {
       cur_c = (int)c;
       cur_g = (int)g;
     }
-    const BsrChunkDesc &cd = p.chunk[c];
+    const BsrChunkDesc &cd = *bsr_desc(p, c);
     const uint4 *src = reinterpret_cast<const uint4 *>(cd.src + src_off);
     uint4 *dst = nullptr;
     if (p.scatter) {
@@ -194,6 +199,252 @@ bsr_install_vec_kernel(const __grid_constant__ BsrInstallParams p) {
   }
   if (cur_c >= 0) bsr_block_flush<THREADS>(sum, p.acc + cur_c * BSR_K_MAX_GROUPS + cur_g, red);
   bsr_install_finish<THREADS>(p);
+}
+
+// ---------------------------------------------------------------------------------------------
+// install, bulk variant: the copy engine of each SM (1-D bulk async copies, no multicast) moves the
+// tiles global -> shared -> global through a ring of shared-memory stages; a producer warp computes
+// addresses and issues the loads, a store warp issues the stores, and four warps sum the tile from
+// shared memory while its store is in flight.
+//
+//   warp 0, producer:  wait empty[s] -> expect_tx(full[s], bytes) -> bulk load tile into stage s
+//   warp 1, storer:    wait full[s]  -> bulk store stage s -> dst; once the store issued two tiles
+//                      earlier has finished reading its stage -> arrive empty[that stage]
+//   warps 2.., sums:   wait full[s]  -> checksum from shared memory -> arrive empty[s]
+//
+// Every wait is bounded by a wall-clock deadline; a wait that gives up raises *err_flag, the CTA
+// stops issuing work, drains what it has in flight and leaves through the common exit.
+// ---------------------------------------------------------------------------------------------
+#define BSR_K_BULK_STAGES 6
+#define BSR_K_BULK_CONSUMER_WARPS 4
+#define BSR_K_BULK_THREADS (32 * (2 + BSR_K_BULK_CONSUMER_WARPS))
+#define BSR_K_BULK_STORE_LAG 2  // stores whose shared-memory reads may still be pending
+#define BSR_K_BULK_SMEM (BSR_K_BULK_STAGES * BSR_K_TILE_MAX)
+#define BSR_K_WAIT_NS 2000000000ull  // 2 s: four orders of magnitude above any legitimate wait
+
+struct BsrStageMeta {
+  uint64_t dst;    // destination address of the tile (0: no store)
+  uint32_t bytes;  // 0 marks the end of this CTA's work
+  uint32_t word0;
+  int32_t c;       // chunk descriptor index
+  int32_t g;       // group
+};
+
+__device__ __forceinline__ uint32_t bsr_smem_u32(const void *p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ uint64_t bsr_globaltimer() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void bsr_mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void bsr_mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void bsr_mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool bsr_mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false if the deadline passed (and raises the error flag).
+__device__ __forceinline__ bool bsr_mbar_wait(uint32_t bar, uint32_t parity, unsigned int *err_flag,
+                                              volatile int *abort_flag) {
+  if (bsr_mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = bsr_globaltimer();
+  for (;;) {
+    if (bsr_mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (bsr_globaltimer() - t0 > BSR_K_WAIT_NS) {
+      *abort_flag = 1;
+      atomicExch(err_flag, 1u);
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ void bsr_bulk_load(uint32_t smem_dst, const void *gsrc, uint32_t bytes,
+                                              uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+          smem_dst),
+      "l"(gsrc), "r"(bytes), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void bsr_bulk_store(uint64_t gdst, uint32_t smem_src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst),
+               "r"(smem_src), "r"(bytes)
+               : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+
+__global__ void __launch_bounds__(BSR_K_BULK_THREADS)
+bsr_install_bulk_kernel(const __grid_constant__ BsrInstallParams p) {
+  extern __shared__ __align__(128) uint8_t stage_mem[];
+  __shared__ __align__(8) uint64_t full_bar[BSR_K_BULK_STAGES];
+  __shared__ __align__(8) uint64_t empty_bar[BSR_K_BULK_STAGES];
+  __shared__ BsrStageMeta meta[BSR_K_BULK_STAGES];
+  __shared__ int last_round[BSR_K_BULK_STAGES];  // last load round issued into each stage, -1 = none
+  __shared__ int abort_flag;
+
+  const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < BSR_K_BULK_STAGES; ++s) {
+      last_round[s] = -1;
+      bsr_mbar_init(bsr_smem_u32(&full_bar[s]), 1);
+      bsr_mbar_init(bsr_smem_u32(&empty_bar[s]), BSR_K_BULK_CONSUMER_WARPS + 1);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+
+  const uint32_t total = p.n_chunks * p.n_tiles;
+  const uint32_t my_tiles = (blockIdx.x < total) ? (total - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+
+  if (warp == 0) {
+    // ---------------- producer ----------------
+    // The address of a tile needs a chain of dependent loads (tile entry -> block table -> tensor
+    // base).  The 32 lanes resolve 32 consecutive tiles of this CTA at once; lane 0 then issues them
+    // in order, taking each tile's values from the lane that resolved it.
+    for (uint32_t base = 0; base < my_tiles; base += 32) {
+      const uint32_t n_mine = base + lane;
+      uint64_t src = 0, dst = 0;
+      uint32_t bytes = 0, word0 = 0, cg = 0;
+      if (n_mine < my_tiles) {
+        const uint32_t w = blockIdx.x + n_mine * gridDim.x;
+        const uint32_t c = w / p.n_tiles, t = w - c * p.n_tiles;
+        const uint4 *tp = reinterpret_cast<const uint4 *>(p.tiles + t);
+        const uint4 t0 = __ldg(tp), t1 = __ldg(tp + 1);
+        const uint32_t g = (t1.y >> 16) & 0xffu;
+        const BsrChunkDesc &cd = *bsr_desc(p, c);
+        if (p.scatter) {
+          const int32_t *table = p.tables[cd.rank * p.n_groups + g];
+          const int32_t phys = __ldg(table + (size_t)cd.chunk * p.blocks_per_chunk[g] + (t1.y >> 24));
+          dst = __ldg(p.tensor_base + (size_t)cd.rank * p.n_tensors + (t1.y & 0xffffu)) +
+                (uint64_t)phys * t1.x + t0.z;
+        }
+        src = reinterpret_cast<uint64_t>(cd.src) + t0.x;
+        bytes = t0.y;
+        word0 = t0.w;
+        cg = (c << 8) | g;
+      }
+      const uint32_t cnt = min(32u, my_tiles - base);
+      int ok = 1;
+      for (uint32_t j = 0; j < cnt && ok; ++j) {
+        const uint64_t src_j = __shfl_sync(0xffffffffu, src, j);
+        const uint64_t dst_j = __shfl_sync(0xffffffffu, dst, j);
+        const uint32_t bytes_j = __shfl_sync(0xffffffffu, bytes, j);
+        const uint32_t word0_j = __shfl_sync(0xffffffffu, word0, j);
+        const uint32_t cg_j = __shfl_sync(0xffffffffu, cg, j);
+        if (lane == 0) {
+          const uint32_t n = base + j;
+          const uint32_t s = n % BSR_K_BULK_STAGES, round = n / BSR_K_BULK_STAGES;
+          if (round > 0 &&
+              !bsr_mbar_wait(bsr_smem_u32(&empty_bar[s]), (round - 1) & 1u, p.err_flag, &abort_flag)) {
+            ok = 0;
+          } else {
+            meta[s].dst = dst_j;
+            meta[s].bytes = bytes_j;
+            meta[s].word0 = word0_j;
+            meta[s].c = (int32_t)(cg_j >> 8);
+            meta[s].g = (int32_t)(cg_j & 0xffu);
+            const uint32_t bar = bsr_smem_u32(&full_bar[s]);
+            bsr_mbar_expect_tx(bar, bytes_j);  // release: the meta writes above are visible to waiters
+            bsr_bulk_load(bsr_smem_u32(stage_mem + (size_t)s * BSR_K_TILE_MAX),
+                          reinterpret_cast<const void *>(src_j), bytes_j, bar);
+            last_round[s] = (int)round;
+          }
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+      }
+      if (!ok) break;
+    }
+  } else if (warp == 1) {
+    // ---------------- storer ----------------
+    if (lane == 0) {
+      uint32_t n = 0;
+      for (; n < my_tiles; ++n) {
+        const uint32_t s = n % BSR_K_BULK_STAGES, round = n / BSR_K_BULK_STAGES;
+        if (!bsr_mbar_wait(bsr_smem_u32(&full_bar[s]), round & 1u, p.err_flag, &abort_flag)) break;
+        if (p.scatter) {
+          bsr_bulk_store(meta[s].dst, bsr_smem_u32(stage_mem + (size_t)s * BSR_K_TILE_MAX),
+                         meta[s].bytes);
+          if (n >= BSR_K_BULK_STORE_LAG) {
+            asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(BSR_K_BULK_STORE_LAG) : "memory");
+            bsr_mbar_arrive(bsr_smem_u32(&empty_bar[(n - BSR_K_BULK_STORE_LAG) % BSR_K_BULK_STAGES]));
+          }
+        } else {
+          bsr_mbar_arrive(bsr_smem_u32(&empty_bar[s]));
+        }
+      }
+      if (p.scatter) {
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        for (uint32_t k = (n > BSR_K_BULK_STORE_LAG ? n - BSR_K_BULK_STORE_LAG : 0); k < n; ++k)
+          bsr_mbar_arrive(bsr_smem_u32(&empty_bar[k % BSR_K_BULK_STAGES]));
+        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // stores complete
+      }
+    }
+  } else {
+    // ---------------- checksum warps ----------------
+    const uint32_t ct = threadIdx.x - 64;  // 0 .. 127
+    uint64_t sum = 0;
+    int cur_c = -1, cur_g = -1;
+    for (uint32_t n = 0; n < my_tiles; ++n) {
+      const uint32_t s = n % BSR_K_BULK_STAGES, round = n / BSR_K_BULK_STAGES;
+      if (!bsr_mbar_wait(bsr_smem_u32(&full_bar[s]), round & 1u, p.err_flag, &abort_flag)) break;
+      const BsrStageMeta m = meta[s];
+      if (m.c != cur_c || m.g != cur_g) {  // warp-uniform
+        if (cur_c >= 0) {
+          sum = bsr_warp_sum(sum);
+          if (lane == 0)
+            atomicAdd((unsigned long long *)(p.acc + cur_c * BSR_K_MAX_GROUPS + cur_g),
+                      (unsigned long long)sum);
+        }
+        sum = 0;
+        cur_c = m.c;
+        cur_g = m.g;
+      }
+      const uint4 *sv = reinterpret_cast<const uint4 *>(stage_mem + (size_t)s * BSR_K_TILE_MAX);
+      const uint32_t nvec = m.bytes >> 4;
+#pragma unroll 4
+      for (uint32_t v = ct; v < nvec; v += 32 * BSR_K_BULK_CONSUMER_WARPS)
+        sum += bsr_ck_vec(sv[v], m.word0 + 4u * v);
+      __syncwarp();
+      if (lane == 0) bsr_mbar_arrive(bsr_smem_u32(&empty_bar[s]));
+    }
+    if (cur_c >= 0) {
+      sum = bsr_warp_sum(sum);
+      if (lane == 0)
+        atomicAdd((unsigned long long *)(p.acc + cur_c * BSR_K_MAX_GROUPS + cur_g),
+                  (unsigned long long)sum);
+    }
+  }
+  __syncthreads();
+  if (abort_flag && threadIdx.x == 0) {
+    // A wait gave up.  Loads this CTA issued may still be landing in its shared memory: give each
+    // stage one more bounded chance to complete before the CTA exits.
+    for (int s = 0; s < BSR_K_BULK_STAGES; ++s) {
+      if (last_round[s] < 0) continue;
+      const uint64_t t0 = bsr_globaltimer();
+      while (!bsr_mbar_try_wait(bsr_smem_u32(&full_bar[s]), (uint32_t)last_round[s] & 1u) &&
+             bsr_globaltimer() - t0 < BSR_K_WAIT_NS / 8) {
+      }
+    }
+  }
+  bsr_install_finish<BSR_K_BULK_THREADS>(p);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -62,6 +62,8 @@ struct bsr_req {
   uint32_t *h_verdict = nullptr;             // pinned, device-visible
   uint64_t *d_ck = nullptr;                  // device aliases of the two arrays above
   uint32_t *d_verdict = nullptr;
+  BsrChunkDesc *h_desc = nullptr;            // pinned: one descriptor per (chunk, rank), batch launches
+  BsrChunkDesc *d_desc = nullptr;            // device copy, uploaded once per restore
   std::vector<uint64_t> bitmap;              // [R*G][words]
   uint32_t words = 0;
   bool restored = false;
@@ -98,6 +100,7 @@ struct bsr_ctx {
   uint64_t *d_acc = nullptr;        // [kLaunchSlots][BATCH][GROUPS]
   unsigned int *d_counters = nullptr;  // [kLaunchSlots] install + [1] probe + [1] err flag
   uint64_t launch_seq = 0;
+  bool bulk_ready = false;  // dynamic shared memory limit of the bulk kernel has been raised
 
   // probe scratch (grown on demand)
   int32_t *d_tok = nullptr;
@@ -109,7 +112,8 @@ struct bsr_ctx {
   uint8_t *ring[BSR_MAX_RANKS] = {};
   uint8_t *dstage[BSR_MAX_RANKS] = {};
   std::vector<cudaEvent_t> ev_h2d, ev_inst, ev_start;  // [R*D]
-  std::vector<cudaEvent_t> ev_batch_start, ev_batch_stop;  // resident mode
+  std::vector<std::pair<cudaEvent_t, cudaEvent_t>> ev_pool;  // launch timing, device-resident restores
+  cudaEvent_t ev_done = nullptr;
 
   // filler pool
   std::vector<std::thread> fillers;
@@ -228,8 +232,20 @@ uint32_t install_grid(const BsrInstallParams &p) {
 }
 
 int launch_install(bsr_ctx *c, const BsrInstallParams &p, cudaStream_t s) {
-  bsr_install_vec_kernel<kInstallThreads, kInstallUnroll>
-      <<<install_grid(p), kInstallThreads, 0, s>>>(p);
+  if (c->cfg.install_variant != BSR_INSTALL_VECTOR) {  // AUTO = bulk: the faster of the two on B200
+    if (!c->bulk_ready) {
+      CU(c, cudaFuncSetAttribute(bsr_install_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 BSR_K_BULK_SMEM));
+      c->bulk_ready = true;
+    }
+    const uint64_t total = (uint64_t)p.n_chunks * p.n_tiles;
+    const uint64_t want = (uint64_t)kSmCount * 2;  // two CTAs of 6 x 16 KiB stages per SM
+    bsr_install_bulk_kernel<<<(uint32_t)(total < want ? total : want), BSR_K_BULK_THREADS,
+                              BSR_K_BULK_SMEM, s>>>(p);
+  } else {
+    bsr_install_vec_kernel<kInstallThreads, kInstallUnroll>
+        <<<install_grid(p), kInstallThreads, 0, s>>>(p);
+  }
   CU(c, cudaGetLastError());
   c->st.kernel_launches++;
   c->st.install_launches++;
@@ -405,10 +421,21 @@ int restore_resident(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_po
                      const std::vector<TierObj> &objs) {
   const uint32_t R = c->cfg.n_ranks, W = c->cfg.window_chunks, N = q->n_adv;
   const uint32_t per_launch = BSR_K_MAX_BATCH / R ? BSR_K_MAX_BATCH / R : 1;
-  std::vector<std::pair<cudaEvent_t, cudaEvent_t>> timing;
   int rc = BSR_OK;
-  cudaEvent_t done;
-  CU(c, cudaEventCreateWithFlags(&done, cudaEventDisableTiming));
+  size_t n_timed = 0;
+  // one descriptor per (chunk, rank) in launch order, uploaded once, ahead of the first launch
+  for (uint32_t i = 0; i < N; ++i)
+    for (uint32_t r = 0; r < R; ++r) {
+      BsrChunkDesc &d = q->h_desc[(size_t)i * R + r];
+      const TierObj &o = objs[(size_t)i * R + r];
+      d.src = o.data;
+      d.chunk = i;
+      d.rank = r;
+      for (uint32_t g = 0; g < BSR_MAX_GROUPS; ++g) d.expect[g] = g < c->G ? o.ck[g] : 0;
+    }
+  CU(c, cudaMemcpyAsync(q->d_desc, q->h_desc, (size_t)N * R * sizeof(BsrChunkDesc),
+                        cudaMemcpyHostToDevice, stream));
+  c->st.h2d_copies++;
   for (uint32_t w0 = 0; w0 < N && rc == BSR_OK; w0 += W) {
     const uint32_t w1 = (w0 + W < N) ? w0 + W : N;
     c->st.windows++;
@@ -421,39 +448,34 @@ int restore_resident(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_po
       p.tables = q->d_table_ptrs;
       p.ck_out = q->d_ck;
       p.verdict = q->d_verdict;
-      for (uint32_t i = b0; i < b1; ++i)
-        for (uint32_t r = 0; r < R; ++r) {
-          BsrChunkDesc &d = p.chunk[p.n_chunks++];
-          const TierObj &o = objs[(size_t)i * R + r];
-          d.src = o.data;
-          d.chunk = i;
-          d.rank = r;
-          for (uint32_t g = 0; g < c->G; ++g) d.expect[g] = o.ck[g];
-        }
-      cudaEvent_t e0 = nullptr, e1 = nullptr;
+      p.batch = q->d_desc + (size_t)b0 * R;
+      p.n_chunks = (b1 - b0) * R;
       if (c->cfg.time_kernels) {
-        CU(c, cudaEventCreate(&e0));
-        CU(c, cudaEventCreate(&e1));
-        CU(c, cudaEventRecord(e0, stream));
+        if (n_timed == c->ev_pool.size()) {
+          cudaEvent_t e0 = nullptr, e1 = nullptr;
+          CU(c, cudaEventCreate(&e0));
+          CU(c, cudaEventCreate(&e1));
+          c->ev_pool.emplace_back(e0, e1);
+        }
+        CU(c, cudaEventRecord(c->ev_pool[n_timed].first, stream));
       }
       rc = launch_install(c, p, stream);
       if (c->cfg.time_kernels) {
-        CU(c, cudaEventRecord(e1, stream));
-        timing.emplace_back(e0, e1);
+        CU(c, cudaEventRecord(c->ev_pool[n_timed].second, stream));
+        ++n_timed;
       }
     }
   }
+  cudaEvent_t done = c->ev_done;
   CU(c, cudaEventRecord(done, stream));
   int wrc = wait_event_deadline(c, done, deadline);
   if (wrc == BSR_ERR_TIMEOUT) {  // kernels are finite: let them finish, then report
     cudaStreamSynchronize(stream);
   }
-  cudaEventDestroy(done);
-  for (auto &pr : timing) {
+  for (size_t k = 0; k < n_timed; ++k) {
     float ms = 0.f;
-    if (cudaEventElapsedTime(&ms, pr.first, pr.second) == cudaSuccess) c->st.install_kernel_ms += ms;
-    cudaEventDestroy(pr.first);
-    cudaEventDestroy(pr.second);
+    if (cudaEventElapsedTime(&ms, c->ev_pool[k].first, c->ev_pool[k].second) == cudaSuccess)
+      c->st.install_kernel_ms += ms;
   }
   if (rc == BSR_OK) rc = wrc;
   if (rc != BSR_OK) return rc;
@@ -596,10 +618,10 @@ int restore_ring(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_point 
       p.ck_out = q->d_ck;
       p.verdict = q->d_verdict;
       p.n_chunks = 1;
-      p.chunk[0].src = stage;
-      p.chunk[0].chunk = i;
-      p.chunk[0].rank = r;
-      for (uint32_t g = 0; g < c->G; ++g) p.chunk[0].expect[g] = o.ck[g];
+      p.one.src = stage;
+      p.one.chunk = i;
+      p.one.rank = r;
+      for (uint32_t g = 0; g < c->G; ++g) p.one.expect[g] = o.ck[g];
       const int lrc = launch_install(c, p, stream);
       e = cudaEventRecord(c->ev_inst[k], stream);
       if (lrc != BSR_OK || e != cudaSuccess) {
@@ -672,6 +694,7 @@ int bsr_ctx_create(const bsr_config *cfg, bsr_ctx **out) {
   bool ok = cudaSetDevice(cfg->device) == cudaSuccess &&
             cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess &&
             cudaStreamCreateWithFlags(&c->own_stream, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaEventCreateWithFlags(&c->ev_done, cudaEventDisableTiming) == cudaSuccess &&
             cudaMalloc(&c->d_acc, acc_bytes) == cudaSuccess &&
             cudaMalloc(&c->d_counters, cnt_bytes) == cudaSuccess &&
             cudaMemset(c->d_acc, 0, acc_bytes) == cudaSuccess &&
@@ -704,6 +727,11 @@ int bsr_ctx_destroy(bsr_ctx *c) {
   for (auto e : c->ev_h2d) cudaEventDestroy(e);
   for (auto e : c->ev_inst) cudaEventDestroy(e);
   for (auto e : c->ev_start) cudaEventDestroy(e);
+  for (auto &pr : c->ev_pool) {
+    cudaEventDestroy(pr.first);
+    cudaEventDestroy(pr.second);
+  }
+  if (c->ev_done) cudaEventDestroy(c->ev_done);
   cudaFree(c->d_tiles);
   cudaFree(c->d_tensor_base);
   cudaFree(c->d_tensor_group);
@@ -847,7 +875,7 @@ int bsr_tier_put(bsr_ctx *c, uint32_t rank, uint64_t key, const void *data, size
     p.ck_out = c->d_put_ck;
     p.verdict = c->d_put_verdict;
     p.n_chunks = 1;
-    p.chunk[0].src = src;
+    p.one.src = src;
     rc = launch_install(c, p, c->own_stream);
     if (rc != BSR_OK) return rc;
     CU(c, cudaStreamSynchronize(c->own_stream));
@@ -1015,6 +1043,10 @@ int bsr_req_create(bsr_ctx *c, const uint64_t *keys, uint32_t n_adv, const int32
       return bail(BSR_ERR_NOMEM, "status arrays");
     memset(q->h_ck, 0, cells * 8);
     memset(q->h_verdict, 0, cells * 4);
+    const size_t n_desc = (size_t)R * n_adv;
+    if (cudaHostAlloc((void **)&q->h_desc, n_desc * sizeof(BsrChunkDesc), cudaHostAllocDefault) != cudaSuccess ||
+        cudaMalloc((void **)&q->d_desc, n_desc * sizeof(BsrChunkDesc)) != cudaSuccess)
+      return bail(BSR_ERR_NOMEM, "descriptor arrays");
   }
   *out = q;
   return BSR_OK;
@@ -1028,6 +1060,8 @@ int bsr_req_release(bsr_ctx *c, bsr_req *q) {
   cudaFree(q->d_table_ptrs);
   if (q->h_ck) cudaFreeHost(q->h_ck);
   if (q->h_verdict) cudaFreeHost(q->h_verdict);
+  if (q->h_desc) cudaFreeHost(q->h_desc);
+  cudaFree(q->d_desc);
   cudaGetLastError();
   delete q;
   return BSR_OK;
@@ -1067,6 +1101,18 @@ int bsr_restore(bsr_ctx *c, bsr_req *q, void *cuda_stream) {
     }
     rc = all_device ? restore_resident(c, q, stream, deadline, objs)
                     : restore_ring(c, q, stream, deadline);
+  }
+  if (N && c->cfg.install_variant != BSR_INSTALL_VECTOR) {
+    // a bounded wait inside the bulk kernel that gave up raised the device-side error flag
+    unsigned int flag = 0;
+    unsigned int *d_flag = c->d_counters + kLaunchSlots + 1;
+    if (cudaMemcpy(&flag, d_flag, sizeof flag, cudaMemcpyDeviceToHost) != cudaSuccess) {
+      if (rc == BSR_OK) rc = fail(c, BSR_ERR_CUDA, "reading the kernel error flag failed");
+    } else if (flag) {
+      cudaMemset(d_flag, 0, sizeof flag);
+      if (rc == BSR_OK || rc == BSR_ERR_CHECKSUM)
+        rc = fail(c, BSR_ERR_TIMEOUT, "a bounded wait inside the install kernel gave up");
+    }
   }
   if (rc == BSR_OK)
     q->restored = true;

@@ -255,3 +255,36 @@ def test_argument_errors_and_empty_request():
     assert B.bsr_req_release(ctx, req) == B.BSR_OK
     assert B.bsr_register(ctx, 0, [(64, 8)], [(0, 32, p)]) == B.BSR_ERR_STATE      # registration in use
     assert B.bsr_ctx_destroy(ctx) == B.BSR_OK
+
+
+# ---------------------------------------------------------------- the bulk-copy install kernel
+@pytest.mark.parametrize("layout_name,R,N,W,location", [
+    ("tiny", 2, 9, 4, 0), ("tiny", 2, 70, 3, 0), ("tiny", 2, 11, 4, 1),
+    ("hetero", 2, 6, 4, 0), ("hetero", 2, 5, 2, 1),
+    ("baseline", 1, 16, 4, 0), ("baseline", 2, 6, 4, 1),
+])
+def test_bulk_install_kernel_matches_oracle(layout_name, R, N, W, location):
+    layout = {"tiny": synth.tiny_layout, "hetero": synth.hetero_layout,
+              "baseline": synth.baseline_layout}[layout_name]()
+    case = Case(layout, R, N, seed=800 + N)
+    ora = run_oracle(case, W)
+    with GpuSide(case, W, location=location, install_variant=2) as gpu:
+        rc, keys, bm, n_hit = gpu.probe()
+        gpu.request(keys, n_hit)
+        assert gpu.restore() == gpu.B.BSR_OK, gpu.B.bsr_last_error(gpu.ctx)
+        _check_success(case, W, gpu, ora, N)
+
+
+def test_bulk_install_kernel_detects_corruption_and_computes_store_checksums():
+    case = Case(synth.hetero_layout(), 2, 4, seed=900)
+    with GpuSide(case, 2, install_variant=2, compute_ck=True) as gpu:
+        B = gpu.B
+        for (r, i), want in case.cks.items():
+            rc, got = B.bsr_tier_checksums(gpu.ctx, r, case.keys[i], case.G)
+            assert rc == B.BSR_OK and [int(x) for x in got] == want
+        rc, keys, bm, n_hit = gpu.probe()
+        gpu.request(keys, n_hit)
+        lo, hi = case.reg.segment(2)
+        case.payload[(1, 3)][lo:hi].view("<u4")[12345] ^= np.uint32(0x10)
+        assert gpu.restore() == B.BSR_ERR_CHECKSUM
+        assert gpu.commit() == 0 and (gpu.bitmap(4) == 0).all()
