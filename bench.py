@@ -31,7 +31,7 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2608_17826_b200 import synth  # noqa: E402
+from paper_2608_17826_b200 import multi, synth  # noqa: E402
 
 WORKLOAD = dict(name="32768-token prefix, 128 chunks x 16,408,576 B, 2 rank slices, W=32, "
                      "baseline 2-group/99-tensor layout, 64-token blocks",
@@ -232,18 +232,14 @@ def timed_steps(torch, dist, world, side, tok, n_tok, salt, tok_on_device, steps
         n_hit, exposed = side.step(tok, n_tok, salt, tok_on_device, stream.cuda_stream)
         ok = ok and n_hit == n_chunks and exposed == n_chunks
         if world > 1:  # request-level commit across GPUs: one word, AND over ranks (Eq. 6)
-            flag = torch.tensor([1 if exposed == n_chunks else 0], device="cuda", dtype=torch.int32)
-            dist.all_reduce(flag, op=dist.ReduceOp.MIN)
-            ok = ok and bool(flag.item())
+            ok = ok and multi.commit_across_ranks(exposed, n_chunks, device="cuda") == n_chunks
     e1.record(stream)
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
     ms = e0.elapsed_time(e1)
     if world > 1:
-        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+        ms = multi.max_over_ranks(ms, device="cuda")
     assert ok, "a step did not expose the full prefix"
     return ms / steps, side.stats()
 
