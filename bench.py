@@ -365,6 +365,50 @@ def run_gpu(args):
     return 0
 
 
+def run_sweep(args):
+    """--sweep: end-to-end restore GB/s vs W and vs fill concurrency on the long prefixes (the
+    paper's window-law and storage-concurrency experiments: throughput moves, peak staging follows
+    W x slot exactly).  The host tier is cyclic: 67 distinct objects per rank, key i -> object i mod 67."""
+    import torch
+    from paper_2608_17826_b200 import build
+    build.build()
+    from paper_2608_17826_b200 import binding as B
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    layout = synth.baseline_layout()
+    R, P, seed = 2, 67, synth.MASTER_SEED
+    objs = {(r, j): synth.chunk_payload(layout, r, j, seed=seed).copy() for r in range(R) for j in range(P)}
+    h2d = measure_h2d(torch, dev, layout.chunk_bytes)
+    plan = [(N, W, 0) for N in (512, 1024) for W in (8, 16, 32, 64)] + [(512, 32, lc) for lc in (1, 2, 4, 8, 16)]
+    for N, W, lc in plan:
+        tok = synth.tokens(N * 256, seed=seed + N)
+        payload = {(r, i): objs[(r, i % P)] for r in range(R) for i in range(N)}
+        side = Side(B, torch, dev, layout, R, N, W, payload, B.BSR_LOC_HOST, load_concurrency=lc,
+                    dev_staging_depth=args.depth, install_variant=args.variant)
+        rc, keys, _, _ = B.bsr_probe(side.ctx, tok, len(tok), seed, False)
+        # stamp checksums once per distinct object, reuse them for the other keys
+        cks = {}
+        for (r, i), o in payload.items():
+            if (r, i % P) not in cks:
+                assert B.bsr_tier_put(side.ctx, r, keys[i], o, o.size, None, B.BSR_LOC_HOST) == B.BSR_OK
+                cks[(r, i % P)] = B.bsr_tier_checksums(side.ctx, r, keys[i], layout.n_groups)[1]
+            else:
+                assert B.bsr_tier_put(side.ctx, r, keys[i], o, o.size, cks[(r, i % P)], B.BSR_LOC_HOST) == B.BSR_OK
+        ms, st = timed_steps(torch, None, 1, side, tok, len(tok), seed, False, 3, 3, N)
+        nbytes = R * N * layout.chunk_bytes
+        print(json.dumps({"sweep": True, "chunks": N, "W": W, "load_concurrency": lc or "auto",
+                          "restore_GBps": nbytes / ms / 1e6, "per_rank_GBps": nbytes / ms / 1e6 / R,
+                          "restore_seconds": ms / 1e3, "frac_of_h2d_link": nbytes / ms / 1e6 / h2d,
+                          "h2d_link_GBps_measured": h2d, "windows_per_restore": int(st.windows) // 3,
+                          "peak_staging_bytes_per_rank": int(st.peak_staging_bytes[0]),
+                          "staging_residual_bytes": int(st.peak_staging_bytes[0]) - W * int(st.slot_bytes)}),
+              flush=True)
+        side.close()
+        del side
+        torch.cuda.empty_cache()
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -375,10 +419,13 @@ def main():
     ap.add_argument("--depth", type=int, default=4)
     ap.add_argument("--variant", type=int, default=0, help="install kernel: 0 auto, 1 vector, 2 bulk copy")
     ap.add_argument("--chunks", type=int, default=0, help="prefix length in chunks (default: the workload's 128)")
+    ap.add_argument("--sweep", action="store_true", help="e2e GB/s vs W and vs fill concurrency (long prefixes)")
     ap.add_argument("--resident-only", action="store_true", help="small profiling runs: skip e2e and CPU legs")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
+    if args.sweep:
+        return run_sweep(args)
     return run_reference(args) if args.impl == "reference" else run_gpu(args)
 
 
