@@ -36,7 +36,7 @@ from paper_2608_17826_b200 import multi, synth  # noqa: E402
 WORKLOAD = dict(name="32768-token prefix, 128 chunks x 16,408,576 B, 2 rank slices, W=32, "
                      "baseline 2-group/99-tensor layout, 64-token blocks",
                 n_chunks=128, n_ranks=2, W=32)
-NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = 1.959  # profiles/install_bulk_kernel_64chunk_launch.md
+NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = 1.957  # profiles/install_bulk_kernel_64chunk_launch.md
 METRIC, UNIT = "restore GB/s (all rank slices; per-rank = value / rank slices)", "GB/s"
 
 
@@ -321,8 +321,9 @@ def run_gpu(args):
     e2e_value = world * step_bytes / (ms_e2e / 1e3) / 1e9
     per_launch_payload = step_bytes * args.steps / max(1, k_launches)
     achieved = 2 * per_launch_payload / (k_ms / 1e3) / 1e9 if k_ms > 0 else None
-    # dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of a launch of this very size
-    # (64 chunk descriptors): 1.0506 GB + 1.0066 GB for 1.0501 GB of payload, i.e. 1.959 B/B.
+    # dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of a smaller launch
+    # (64 chunk descriptors, a quarter of the timed launch; traffic grows in proportion to the
+    # descriptors processed): 1.0503 GB + 1.0050 GB for 1.0501 GB of payload, i.e. 1.957 B/B.
     traffic = NCU_DRAM_BYTES_PER_PAYLOAD_BYTE * per_launch_payload
 
     # ---- CPU oracle on a bounded sample -----------------------------------------------------

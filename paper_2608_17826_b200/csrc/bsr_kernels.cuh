@@ -8,7 +8,7 @@
 #include <stdint.h>
 
 #define BSR_K_MAX_GROUPS 8
-#define BSR_K_MAX_BATCH 64        // chunk descriptors per install launch
+#define BSR_K_MAX_BATCH 256       // chunk descriptors per install launch
 #define BSR_K_TILE_MAX 16384u     // largest tile in bytes (one bulk-copy stage)
 #define BSR_K_PHI 0x9E3779B97F4A7C15ull
 
@@ -274,17 +274,24 @@ __device__ __forceinline__ bool bsr_mbar_wait(uint32_t bar, uint32_t parity, uns
     }
   }
 }
+__device__ __forceinline__ uint64_t bsr_policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
 __device__ __forceinline__ void bsr_bulk_load(uint32_t smem_dst, const void *gsrc, uint32_t bytes,
-                                              uint32_t bar) {
+                                                   uint32_t bar, uint64_t pol) {
   asm volatile(
-      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-          smem_dst),
-      "l"(gsrc), "r"(bytes), "r"(bar)
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, "
+      "[%3], %4;" ::"r"(smem_dst),
+      "l"(gsrc), "r"(bytes), "r"(bar), "l"(pol)
       : "memory");
 }
-__device__ __forceinline__ void bsr_bulk_store(uint64_t gdst, uint32_t smem_src, uint32_t bytes) {
-  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst),
-               "r"(smem_src), "r"(bytes)
+__device__ __forceinline__ void bsr_bulk_store(uint64_t gdst, uint32_t smem_src, uint32_t bytes,
+                                                    uint64_t pol) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;" ::"l"(
+                   gdst),
+               "r"(smem_src), "r"(bytes), "l"(pol)
                : "memory");
   asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
@@ -311,6 +318,8 @@ bsr_install_bulk_kernel(const __grid_constant__ BsrInstallParams p) {
   }
   __syncthreads();
 
+  // every byte is read once and written once: mark both streams evict-first in L2
+  const uint64_t pol = bsr_policy_evict_first();
   const uint32_t total = p.n_chunks * p.n_tiles;
   const uint32_t my_tiles = (blockIdx.x < total) ? (total - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
 
@@ -364,7 +373,7 @@ bsr_install_bulk_kernel(const __grid_constant__ BsrInstallParams p) {
             const uint32_t bar = bsr_smem_u32(&full_bar[s]);
             bsr_mbar_expect_tx(bar, bytes_j);  // release: the meta writes above are visible to waiters
             bsr_bulk_load(bsr_smem_u32(stage_mem + (size_t)s * BSR_K_TILE_MAX),
-                          reinterpret_cast<const void *>(src_j), bytes_j, bar);
+                          reinterpret_cast<const void *>(src_j), bytes_j, bar, pol);
             last_round[s] = (int)round;
           }
         }
@@ -381,7 +390,7 @@ bsr_install_bulk_kernel(const __grid_constant__ BsrInstallParams p) {
         if (!bsr_mbar_wait(bsr_smem_u32(&full_bar[s]), round & 1u, p.err_flag, &abort_flag)) break;
         if (p.scatter) {
           bsr_bulk_store(meta[s].dst, bsr_smem_u32(stage_mem + (size_t)s * BSR_K_TILE_MAX),
-                         meta[s].bytes);
+                         meta[s].bytes, pol);
           if (n >= BSR_K_BULK_STORE_LAG) {
             asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(BSR_K_BULK_STORE_LAG) : "memory");
             bsr_mbar_arrive(bsr_smem_u32(&empty_bar[(n - BSR_K_BULK_STORE_LAG) % BSR_K_BULK_STAGES]));

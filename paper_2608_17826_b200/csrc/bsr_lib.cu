@@ -240,8 +240,8 @@ int launch_install(bsr_ctx *c, const BsrInstallParams &p, cudaStream_t s) {
     }
     const uint64_t total = (uint64_t)p.n_chunks * p.n_tiles;
     const uint64_t want = (uint64_t)kSmCount * 2;  // two CTAs of 6 x 16 KiB stages per SM
-    bsr_install_bulk_kernel<<<(uint32_t)(total < want ? total : want), BSR_K_BULK_THREADS,
-                              BSR_K_BULK_SMEM, s>>>(p);
+    const uint32_t grid = (uint32_t)(total < want ? total : want);
+    bsr_install_bulk_kernel<<<grid, BSR_K_BULK_THREADS, BSR_K_BULK_SMEM, s>>>(p);
   } else {
     bsr_install_vec_kernel<kInstallThreads, kInstallUnroll>
         <<<install_grid(p), kInstallThreads, 0, s>>>(p);
@@ -436,10 +436,12 @@ int restore_resident(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_po
   CU(c, cudaMemcpyAsync(q->d_desc, q->h_desc, (size_t)N * R * sizeof(BsrChunkDesc),
                         cudaMemcpyHostToDevice, stream));
   c->st.h2d_copies++;
-  for (uint32_t w0 = 0; w0 < N && rc == BSR_OK; w0 += W) {
-    const uint32_t w1 = (w0 + W < N) ? w0 + W : N;
-    c->st.windows++;
-    for (uint32_t b0 = w0; b0 < w1 && rc == BSR_OK; b0 += per_launch) {
+  // Nothing is staged for device-resident objects, so a window bounds nothing here: it is counted
+  // (K = ceil(N / W)) and the launches take as many chunks as the kernel's scratch allows.
+  c->st.windows += (N + W - 1) / W;
+  {
+    const uint32_t w1 = N;
+    for (uint32_t b0 = 0; b0 < w1 && rc == BSR_OK; b0 += per_launch) {
       const uint32_t b1 = (b0 + per_launch < w1) ? b0 + per_launch : w1;
       BsrInstallParams p{};
       fill_params(c, p, (uint32_t)(c->launch_seq++ % kLaunchSlots));

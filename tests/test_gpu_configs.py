@@ -1,8 +1,8 @@
 """The five workload configurations at their full sizes on a B200, against the oracle.
 
 Configuration 2 (the benchmarked one) is fully materialised and every paged byte is compared,
-in both launch configurations the benchmark times (device-resident tier: 64 chunk descriptors
-per install launch; host tier: ring + one chunk per launch).  Configurations 3-5 move 8-67 GB
+in both launch configurations the benchmark times (device-resident tier: all 256 chunk
+descriptors in one install launch; host tier: ring + one chunk per launch).  Configurations 3-5 move 8-67 GB
 per rank; there the host tier is cyclic (P distinct seeded objects per rank, P prime and > W,
 key i -> object i mod P) so that the oracle can checksum every object, and the result is checked
 through: every (rank, group, chunk) checksum the install kernel computed == the oracle's checksum
