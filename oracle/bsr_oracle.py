@@ -347,3 +347,61 @@ def invalidate(reg: Registration, req: Request, paged, scrub: bool):
             for l, (g, _) in enumerate(reg.tensors):
                 for blk in req.block_tables[r][g]:
                     paged[r][l][blk] = 0
+
+
+# --------------------------------------------------------------------------------------
+# request-level recovery  (Section 3 "Recover without re-entering the same fault";
+# Section 6.4 failure outcomes: lower valid tier when available, otherwise zero external reuse)
+# --------------------------------------------------------------------------------------
+@dataclass
+class Engine:
+    """The reusable tiers of one engine in priority order (tier 0 first, e.g. remote DRAM, then a
+    lower tier such as local SSD), their availability, and the force-local markers."""
+
+    tiers: list[list[Tier]]                 # [tier][rank]
+    available: list[bool]
+    force_local: set = field(default_factory=set)
+
+
+def probe_request(eng: Engine, request_id: int, tok: np.ndarray, salt: int, reg_id: int):
+    """Request-scoped probe.  Returns (keys, hit, n_hit, tier).
+    A request carrying the force-local marker reports zero external tokens without consulting any
+    tier (tier = -1).  Otherwise every available tier is probed as in `probe`; the request is
+    served by ONE tier, the one with the longest complete prefix, the higher-priority tier on a
+    tie.  With no available tier or no hit, n_hit = 0 and tier = -1."""
+    keys = prefix_keys(chunk_digests(tok, salt), salt, reg_id)
+    none = np.zeros(len(keys), dtype=bool)
+    if request_id in eng.force_local:
+        return keys, none, 0, -1
+    best_tier, best_n, best_hit = -1, 0, none
+    for t, ranks in enumerate(eng.tiers):
+        if not eng.available[t]:
+            continue
+        hit = np.array([all(rk.contains(k) for rk in ranks) for k in keys], dtype=bool)
+        n = int(np.argmin(hit)) if not hit.all() else len(hit)
+        if n > best_n:
+            best_tier, best_n, best_hit = t, n, hit
+    return keys, best_hit, best_n, best_tier
+
+
+def restore_request(eng: Engine, request_id: int, tier: int, reg: Registration, req: Request,
+                    paged, W: int, fetch_fault=None):
+    """Restore of a bound request from the tier the probe chose.  A tier that has become
+    unavailable fails the retrieve as a transfer error.  Any failure installs the force-local
+    marker for the request, so that its next probe reports zero external tokens."""
+    if tier < 0 or tier >= len(eng.tiers):
+        return ERR_INVALID, Stats([0] * req.n_ranks, [0] * req.n_ranks, [0] * req.n_ranks)
+    if not eng.available[tier]:
+        req.valid[:] = False
+        req.restored, req.failed = False, True
+        eng.force_local.add(request_id)
+        return ERR_TRANSFER, Stats([0] * req.n_ranks, [0] * req.n_ranks, [0] * req.n_ranks)
+    status, st = restore(reg, eng.tiers[tier], req, paged, W, fetch_fault=fetch_fault)
+    if status != OK:
+        eng.force_local.add(request_id)
+    return status, st
+
+
+def request_done(eng: Engine, request_id: int):
+    """Successful RUNNING admission or request teardown removes the marker."""
+    eng.force_local.discard(request_id)

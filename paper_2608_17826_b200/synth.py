@@ -35,10 +35,9 @@ def _rng(*key: int) -> np.random.Generator:
 class Layout:
     """A registration geometry: allocator groups and the tensors registered in each.
 
-    groups:  list of (block_tokens, n_logical_blocks_hint) is NOT stored here; only the
-             per-group block size in tokens.  Pool sizes depend on the prefix length and
-             are chosen by `pool_blocks`.
-    tensors: list of (group, bytes_per_token) in registration order, group-major.
+    block_tokens: tokens per paged block of each group (pool sizes depend on the prefix length
+                  and come from `pool_blocks`).
+    tensors:      (group, bytes_per_token) in registration order, group-major.
     """
 
     name: str
@@ -65,11 +64,13 @@ def baseline_layout() -> Layout:
     return Layout("baseline-2group-99tensor", [64, 64], tensors)
 
 
-def hetero_layout(seed: int = MASTER_SEED) -> Layout:
+def hetero_layout(seed: int = MASTER_SEED, bytes_per_token: int = 64096,
+                  name: str = "hetero-3group-170tensor") -> Layout:
     """170 registered tensors of heterogeneous per-token sizes (multiples of 16 B) that sum
-    to 64,096 B/token, in three allocator groups with 64-, 16- and 64-token blocks.
-    Tensors [0,90) -> group 0, [90,140) -> group 1, [140,170) -> group 2."""
-    n, units_total = 170, 64096 // 16
+    to `bytes_per_token` (64,096 by default), in three allocator groups with 64-, 16- and
+    64-token blocks.  Tensors [0,90) -> group 0, [90,140) -> group 1, [140,170) -> group 2."""
+    assert bytes_per_token % 16 == 0
+    n, units_total = 170, bytes_per_token // 16
     rng = _rng(seed, _TAG_SIZES)
     # skewed weights: a few wide tensors, many narrow ones
     w = 1.0 + rng.integers(0, 64, size=n).astype(np.float64) ** 2 / 64.0
@@ -80,7 +81,14 @@ def hetero_layout(seed: int = MASTER_SEED) -> Layout:
     assert int(units.sum()) == units_total
     groups = [0] * 90 + [1] * 50 + [2] * 30
     tensors = [(g, int(16 * u)) for g, u in zip(groups, units)]
-    return Layout("hetero-3group-170tensor", [64, 16, 64], tensors)
+    return Layout(name, [64, 16, 64], tensors)
+
+
+def mtp_on_layout(seed: int = MASTER_SEED) -> Layout:
+    """The paper's MTP-on registration size: 170 tensors accounting to 16,633,856 B per chunk
+    (64,976 B/token; Section 6.4 reports 532,283,392 B = 32 x 16,633,856 at W = 32).  The paper
+    gives only the tensor count and the total, so the individual sizes are seeded like `hetero_layout`."""
+    return hetero_layout(seed=seed + 1, bytes_per_token=64976, name="mtp-on-3group-170tensor")
 
 
 def tiny_layout() -> Layout:

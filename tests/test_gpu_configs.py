@@ -179,10 +179,14 @@ def test_config3_window_sweep_staging_law(N):
             gpu.close()
 
 
-@pytest.mark.parametrize("layout_name", ["baseline", "hetero"])
+@pytest.mark.parametrize("layout_name", ["baseline", "hetero", "mtp_on"])
 def test_config4_2048_chunks(layout_name):
-    layout = synth.baseline_layout() if layout_name == "baseline" else synth.hetero_layout()
-    N, W = 2048, 32
+    """2,048 chunks of the baseline and the 170-tensor layouts; and the paper's MTP-on registration
+    size (16,633,856 B/chunk) at its own length of 524,032 tokens = 2,047 chunks, a prefix that is not a
+    multiple of W, where the paper prints a peak of 532,283,392 B/rank."""
+    layout = {"baseline": synth.baseline_layout, "hetero": synth.hetero_layout,
+              "mtp_on": synth.mtp_on_layout}[layout_name]()
+    N, W = (2047 if layout_name == "mtp_on" else 2048), 32
     case = CyclicCase(layout, 2, N, P=67, seed=4004)
     gpu = BigGpu(case, W)
     try:
@@ -192,7 +196,11 @@ def test_config4_2048_chunks(layout_name):
         assert gpu.B.bsr_restore(gpu.ctx, gpu.req) == gpu.B.BSR_OK, gpu.B.bsr_last_error(gpu.ctx)
         gpu.check_success(W, N)
         st = gpu.B.bsr_get_stats(gpu.ctx)[1]
-        assert st.bytes_installed[0] == 33_604_763_648 and st.peak_staging_bytes[0] == 525_074_432
+        if layout_name == "mtp_on":
+            assert st.peak_staging_bytes[0] == int(read_golden("paper_capacity.txt")["mtp_on_peak_w32"])
+            assert st.bytes_installed[0] == 2047 * 16_633_856 and st.windows == 64
+        else:
+            assert st.bytes_installed[0] == 33_604_763_648 and st.peak_staging_bytes[0] == 525_074_432
     finally:
         gpu.close()
 

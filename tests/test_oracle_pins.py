@@ -161,6 +161,8 @@ def test_baseline_registration_matches_the_papers_coefficient():
     assert O.Registration([64], [(0, 64976)]).slot_bytes * 32 == int(g["mtp_on_peak_w32"])
     hl = _reg(synth.hetero_layout())
     assert hl.chunk_bytes == c and len(hl.tensors) == 170 and hl.n_groups == 3
+    ml = _reg(synth.mtp_on_layout())
+    assert len(ml.tensors) == 170 and 32 * ml.slot_bytes == int(g["mtp_on_peak_w32"])
 
 
 def test_slot_rounding_rule():
