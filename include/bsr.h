@@ -37,6 +37,8 @@ extern "C" {
 #define BSR_CHUNK_TOKENS 256u /* Section 4 "System topology": the chunk is 256 tokens        */
 #define BSR_MAX_GROUPS 8u     /* allocator groups per registration                             */
 #define BSR_MAX_RANKS 8u      /* TP rank slices per context                                    */
+#define BSR_MAX_TIERS 4u      /* reusable tiers in priority order: 0 first (e.g. remote DRAM),
+                                 then lower tiers (e.g. local SSD)                              */
 
 enum {
   BSR_OK = 0,
@@ -106,6 +108,7 @@ typedef struct bsr_stats {
   uint64_t kernel_launches;                     /* kernels of this library launched                  */
   uint64_t h2d_copies;                          /* cudaMemcpyAsync calls issued                      */
   uint64_t install_launches;                    /* install kernel launches                           */
+  uint64_t bytes_restored_by_tier[BSR_MAX_TIERS]; /* verified and installed, by source tier          */
   double install_kernel_ms;                     /* sum of their device durations (time_kernels)      */
   double last_restore_ms;                       /* host wall time of the last bsr_restore            */
 } bsr_stats;
@@ -244,6 +247,38 @@ enum {
  * and host threads only; the GPU is never made to fault, trap or spin. */
 int bsr_test_inject(bsr_ctx *ctx, int kind, uint32_t rank, uint32_t group, uint32_t chunk,
                     uint64_t seed);
+
+/* ---- request-level recovery (Section 3 "Recover without re-entering the same fault";
+ *      Section 6.4: lower valid tier when available, otherwise zero external reuse) ---------- */
+
+/* bsr_tier_put / bsr_tier_remove act on tier 0.  These address any tier 0..BSR_MAX_TIERS-1. */
+int bsr_tier_put_at(bsr_ctx *ctx, uint32_t tier, uint32_t rank, uint64_t key, const void *data,
+                    size_t len, const uint64_t *group_ck, int location);
+int bsr_tier_remove_at(bsr_ctx *ctx, uint32_t tier, uint32_t rank, uint64_t key);
+
+/* Marks a tier reachable (default) or unreachable.  An unreachable tier is skipped by
+ * bsr_probe_request, and a restore bound to it fails closed with BSR_ERR_TRANSFER. */
+int bsr_tier_set_available(bsr_ctx *ctx, uint32_t tier, int available);
+
+/* Request-scoped probe: same keys and bitmap semantics as bsr_probe, but
+ *   - if request_id carries the force-local marker, zero external chunks are reported and no tier
+ *     is consulted (tier_out = -1): the request re-enters local prefill;
+ *   - otherwise every available tier is probed and ONE tier serves the request: the one with the
+ *     longest complete prefix, the higher-priority (lower-numbered) tier on a tie.  hit_bitmap_out
+ *     is that tier's raw hit bitmap; tier_out = -1 when nothing is reusable. */
+int bsr_probe_request(bsr_ctx *ctx, uint64_t request_id, const int32_t *tok, size_t n_tok,
+                      int tok_on_device, uint64_t salt, uint64_t *keys_out, uint64_t *hit_bitmap_out,
+                      uint32_t *n_hit_chunks, int *tier_out);
+
+/* Binds a request object to the engine's request identity and to the tier its probe chose.  A
+ * bound request whose restore fails (any error) installs the force-local marker for request_id.
+ * Unbound requests (the default) restore from tier 0 and leave no marker. */
+int bsr_req_bind(bsr_ctx *ctx, bsr_req *req, uint64_t request_id, uint32_t tier);
+
+/* Removes the marker: call after the request reached RUNNING admission or was torn down. */
+int bsr_request_done(bsr_ctx *ctx, uint64_t request_id);
+
+int bsr_request_is_force_local(bsr_ctx *ctx, uint64_t request_id, int *out);
 
 /* ---- allocation-free prefix keys ----------------------------------------------------------- */
 

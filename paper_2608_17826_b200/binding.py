@@ -31,8 +31,10 @@ EXPORTS = [
     "bsr_tier_put", "bsr_tier_remove", "bsr_tier_checksums", "bsr_probe", "bsr_req_create",
     "bsr_req_release", "bsr_restore", "bsr_commit", "bsr_invalidate", "bsr_req_bitmap",
     "bsr_req_checksums", "bsr_get_stats", "bsr_reset_stats", "bsr_test_inject",
-    "bsr_probe_keys_noalloc",
+    "bsr_probe_keys_noalloc", "bsr_tier_put_at", "bsr_tier_remove_at", "bsr_tier_set_available",
+    "bsr_probe_request", "bsr_req_bind", "bsr_request_done", "bsr_request_is_force_local",
 ]
+BSR_MAX_TIERS = 4
 BSR_NOALLOC_MAX_CHUNKS = 8192
 
 
@@ -60,6 +62,7 @@ class bsr_stats(C.Structure):
                 ("slot_bytes", C.c_uint64), ("dev_aux_bytes", C.c_uint64), ("windows", C.c_uint64),
                 ("tier_bytes_read_by_probe", C.c_uint64), ("kernel_launches", C.c_uint64),
                 ("h2d_copies", C.c_uint64), ("install_launches", C.c_uint64),
+                ("bytes_restored_by_tier", C.c_uint64 * 4),
                 ("install_kernel_ms", C.c_double), ("last_restore_ms", C.c_double)]
 
 
@@ -90,6 +93,13 @@ def _load() -> C.CDLL:
         "bsr_reset_stats": [vp],
         "bsr_test_inject": [vp, i32, u32, u32, u32, u64],
         "bsr_probe_keys_noalloc": [i32, vp, C.c_size_t, u64, u64, vp, vp],
+        "bsr_tier_put_at": [vp, u32, u32, u64, vp, C.c_size_t, vp, i32],
+        "bsr_tier_remove_at": [vp, u32, u32, u64],
+        "bsr_tier_set_available": [vp, u32, i32],
+        "bsr_probe_request": [vp, u64, vp, C.c_size_t, i32, u64, vp, vp, C.POINTER(u32), C.POINTER(i32)],
+        "bsr_req_bind": [vp, vp, u64, u32],
+        "bsr_request_done": [vp, u64],
+        "bsr_request_is_force_local": [vp, u64, C.POINTER(i32)],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -231,3 +241,43 @@ def bsr_probe_keys_noalloc(device: int, d_tok: int, n_tok: int, salt: int, reg_i
     """Prefix keys for callers that must not allocate: device pointers in, device pointer out,
     enqueued on `cuda_stream`; at most BSR_NOALLOC_MAX_CHUNKS chunks (see include/bsr.h)."""
     return lib.bsr_probe_keys_noalloc(device, d_tok, n_tok, int(salt), int(reg_id), d_keys_out, cuda_stream)
+
+
+# ---- request-level recovery ----------------------------------------------------------------------
+def bsr_tier_put_at(ctx, tier: int, rank: int, key: int, data, nbytes: int, group_ck=None,
+                    location: int = BSR_LOC_HOST) -> int:
+    ck = None if group_ck is None else np.ascontiguousarray(group_ck, dtype=np.uint64)
+    return lib.bsr_tier_put_at(ctx, tier, rank, int(key), _ptr(data), nbytes, _ptr(ck), location)
+
+
+def bsr_tier_remove_at(ctx, tier: int, rank: int, key: int) -> int:
+    return lib.bsr_tier_remove_at(ctx, tier, rank, int(key))
+
+
+def bsr_tier_set_available(ctx, tier: int, available: bool) -> int:
+    return lib.bsr_tier_set_available(ctx, tier, int(available))
+
+
+def bsr_probe_request(ctx, request_id: int, tok, n_tok: int, salt: int, tok_on_device: bool = False):
+    """Returns (rc, keys[N], hit_bitmap[ceil(N/64)], n_hit_chunks, tier)."""
+    n = n_tok // BSR_CHUNK_TOKENS
+    keys = np.zeros(n, dtype=np.uint64)
+    bitmap = np.zeros((n + 63) // 64, dtype=np.uint64)
+    n_hit, tier = C.c_uint32(0), C.c_int(-1)
+    rc = lib.bsr_probe_request(ctx, int(request_id), _ptr(tok), n_tok, int(tok_on_device), int(salt),
+                               _ptr(keys), _ptr(bitmap), C.byref(n_hit), C.byref(tier))
+    return rc, keys, bitmap, n_hit.value, tier.value
+
+
+def bsr_req_bind(ctx, req, request_id: int, tier: int) -> int:
+    return lib.bsr_req_bind(ctx, req, int(request_id), tier)
+
+
+def bsr_request_done(ctx, request_id: int) -> int:
+    return lib.bsr_request_done(ctx, int(request_id))
+
+
+def bsr_request_is_force_local(ctx, request_id: int):
+    out = C.c_int(0)
+    rc = lib.bsr_request_is_force_local(ctx, int(request_id), C.byref(out))
+    return rc, bool(out.value)

@@ -16,6 +16,7 @@
 #include <string>
 #include <thread>
 #include <unordered_map>
+#include <unordered_set>
 #include <vector>
 
 #include "bsr_kernels.cuh"
@@ -68,6 +69,9 @@ struct bsr_req {
   uint32_t words = 0;
   bool restored = false;
   bool failed = false;
+  uint64_t request_id = 0;  // engine's request identity (bsr_req_bind); 0 = unbound
+  uint32_t tier = 0;        // the one tier this request is served from
+  bool bound = false;
 };
 
 struct bsr_ctx {
@@ -90,7 +94,9 @@ struct bsr_ctx {
   uint32_t *d_tensor_group = nullptr, *d_tensor_run = nullptr;
 
   // tier + index
-  std::unordered_map<uint64_t, TierObj> tier[BSR_MAX_RANKS];
+  std::unordered_map<uint64_t, TierObj> tier[BSR_MAX_TIERS][BSR_MAX_RANKS];
+  bool tier_available[BSR_MAX_TIERS] = {true, true, true, true};
+  std::unordered_set<uint64_t> force_local;  // request ids whose next probe must report zero
   uint8_t *d_put_stage = nullptr;
   uint64_t *h_put_ck = nullptr, *d_put_ck = nullptr;  // pinned [G] sums + verdict dump
   uint32_t *h_put_verdict = nullptr, *d_put_verdict = nullptr;
@@ -309,18 +315,22 @@ void filler_main(bsr_ctx *c) {
     int state = 1;
     TierObj obj{};
     if (!c->fill_abort.load(std::memory_order_acquire)) {
-      bool found = false;
+      bool found = false, tier_down = false;
       {
         std::lock_guard<std::mutex> g(c->mu);
-        auto it = c->tier[r].find(req->keys[i]);
-        if (it != c->tier[r].end()) {
+        auto &index = c->tier[req->tier][r];
+        auto it = index.find(req->keys[i]);
+        if (it != index.end()) {
           obj = it->second;
           found = true;
         }
+        if (!c->tier_available[req->tier]) tier_down = true;
       }
       const Inject inj = c->inject;
       const bool hit = inj.kind != BSR_INJECT_NONE && inj.rank == r && inj.chunk == i;
-      if (!found) {
+      if (tier_down) {
+        state = BSR_ERR_TRANSFER;  // the tier went away after the probe
+      } else if (!found) {
         state = BSR_ERR_MISSING;
       } else if (hit && inj.kind == BSR_INJECT_FILL_ERROR) {
         state = BSR_ERR_TRANSFER;
@@ -837,7 +847,12 @@ int bsr_chunk_bytes(bsr_ctx *c, uint64_t *chunk_bytes, uint64_t *slot_bytes) {
 
 int bsr_tier_put(bsr_ctx *c, uint32_t rank, uint64_t key, const void *data, size_t len,
                  const uint64_t *group_ck, int location) {
-  if (!c || !data) return BSR_ERR_INVALID;
+  return bsr_tier_put_at(c, 0, rank, key, data, len, group_ck, location);
+}
+
+int bsr_tier_put_at(bsr_ctx *c, uint32_t tier, uint32_t rank, uint64_t key, const void *data,
+                    size_t len, const uint64_t *group_ck, int location) {
+  if (!c || !data || tier >= BSR_MAX_TIERS) return BSR_ERR_INVALID;
   if (rank >= c->cfg.n_ranks || (location != BSR_LOC_HOST && location != BSR_LOC_DEVICE))
     return fail(c, BSR_ERR_INVALID, "tier_put: bad rank or location");
   if (c->L == 0) return fail(c, BSR_ERR_STATE, "tier_put before registration");
@@ -884,29 +899,44 @@ int bsr_tier_put(bsr_ctx *c, uint32_t rank, uint64_t key, const void *data, size
     for (uint32_t g = 0; g < c->G; ++g) o.ck[g] = c->h_put_ck[g];
   }
   std::lock_guard<std::mutex> lk(c->mu);
-  c->tier[rank][key] = o;
+  c->tier[tier][rank][key] = o;
   return BSR_OK;
 }
 
 int bsr_tier_remove(bsr_ctx *c, uint32_t rank, uint64_t key) {
-  if (!c || rank >= c->cfg.n_ranks) return BSR_ERR_INVALID;
+  return bsr_tier_remove_at(c, 0, rank, key);
+}
+
+int bsr_tier_remove_at(bsr_ctx *c, uint32_t tier, uint32_t rank, uint64_t key) {
+  if (!c || rank >= c->cfg.n_ranks || tier >= BSR_MAX_TIERS) return BSR_ERR_INVALID;
   std::lock_guard<std::mutex> lk(c->mu);
-  c->tier[rank].erase(key);
+  c->tier[tier][rank].erase(key);
+  return BSR_OK;
+}
+
+int bsr_tier_set_available(bsr_ctx *c, uint32_t tier, int available) {
+  if (!c || tier >= BSR_MAX_TIERS) return BSR_ERR_INVALID;
+  std::lock_guard<std::mutex> lk(c->mu);
+  c->tier_available[tier] = available != 0;
   return BSR_OK;
 }
 
 int bsr_tier_checksums(bsr_ctx *c, uint32_t rank, uint64_t key, uint64_t *out) {
   if (!c || !out || rank >= c->cfg.n_ranks) return BSR_ERR_INVALID;
   std::lock_guard<std::mutex> lk(c->mu);
-  auto it = c->tier[rank].find(key);
-  if (it == c->tier[rank].end()) return BSR_ERR_MISSING;
+  auto it = c->tier[0][rank].find(key);
+  if (it == c->tier[0][rank].end()) return BSR_ERR_MISSING;
   for (uint32_t g = 0; g < c->G; ++g) out[g] = it->second.ck[g];
   return BSR_OK;
 }
 
-int bsr_probe(bsr_ctx *c, const int32_t *tok, size_t n_tok, int tok_on_device, uint64_t salt,
-              uint64_t *keys_out, uint64_t *hit_bitmap_out, uint32_t *n_hit_chunks) {
+// Shared by bsr_probe (tier 0, no request identity) and bsr_probe_request (all available tiers,
+// force-local marker).  request_scoped selects the second behaviour.
+static int probe_impl(bsr_ctx *c, bool request_scoped, uint64_t request_id, const int32_t *tok,
+                      size_t n_tok, int tok_on_device, uint64_t salt, uint64_t *keys_out,
+                      uint64_t *hit_bitmap_out, uint32_t *n_hit_chunks, int *tier_out) {
   if (!c || (!tok && n_tok) || !n_hit_chunks) return BSR_ERR_INVALID;
+  if (tier_out) *tier_out = -1;
   const size_t N = n_tok / BSR_CHUNK_TOKENS;
   if (N > (1u << 24)) return fail(c, BSR_ERR_INVALID, "probe: more than 2^24 chunks");
   if (tok_on_device && (reinterpret_cast<uintptr_t>(tok) & 15u))
@@ -956,22 +986,75 @@ int bsr_probe(bsr_ctx *c, const int32_t *tok, size_t n_tok, int tok_on_device, u
   CU(c, cudaMemcpyAsync(c->h_keys, c->d_keys, N * 8, cudaMemcpyDeviceToHost, s));
   CU(c, cudaStreamSynchronize(s));
   // index lookup: keys only; no payload byte is read, nothing is pinned or referenced afterwards
-  uint32_t n_hit = 0;
-  bool prefix = true;
-  if (hit_bitmap_out) memset(hit_bitmap_out, 0, (N + 63) / 64 * 8);
+  const size_t words = (N + 63) / 64;
+  if (hit_bitmap_out) memset(hit_bitmap_out, 0, words * 8);
+  uint32_t best_n = 0;
+  int best_tier = -1;
   {
     std::lock_guard<std::mutex> lk(c->mu);
-    for (size_t i = 0; i < N; ++i) {
-      bool hit = true;
-      for (uint32_t r = 0; r < c->cfg.n_ranks && hit; ++r)
-        hit = c->tier[r].find(c->h_keys[i]) != c->tier[r].end();
-      if (hit && hit_bitmap_out) hit_bitmap_out[i / 64] |= 1ull << (i % 64);
-      if (!hit) prefix = false;
-      if (prefix) ++n_hit;
+    const bool forced = request_scoped && c->force_local.count(request_id) != 0;
+    std::vector<uint64_t> bm(words), best_bm(words, 0ull);
+    for (uint32_t t = 0; t < BSR_MAX_TIERS && !forced; ++t) {
+      if (request_scoped ? !c->tier_available[t] : t != 0) continue;
+      std::fill(bm.begin(), bm.end(), 0ull);
+      uint32_t n_hit = 0;
+      bool prefix = true;
+      for (size_t i = 0; i < N; ++i) {
+        bool hit = true;
+        for (uint32_t r = 0; r < c->cfg.n_ranks && hit; ++r)
+          hit = c->tier[t][r].find(c->h_keys[i]) != c->tier[t][r].end();
+        if (hit) bm[i / 64] |= 1ull << (i % 64);
+        if (!hit) prefix = false;
+        if (prefix) ++n_hit;
+      }
+      // one tier serves the request: the longest complete prefix, the higher-priority tier on a tie
+      if (n_hit > best_n || (!request_scoped && t == 0)) {
+        best_n = n_hit;
+        best_tier = n_hit ? (int)t : -1;
+        best_bm = bm;
+      }
     }
+    if (hit_bitmap_out) memcpy(hit_bitmap_out, best_bm.data(), words * 8);
   }
   if (keys_out) memcpy(keys_out, c->h_keys, N * 8);
-  *n_hit_chunks = n_hit;
+  *n_hit_chunks = best_n;
+  if (tier_out) *tier_out = best_tier;
+  return BSR_OK;
+}
+
+int bsr_probe(bsr_ctx *c, const int32_t *tok, size_t n_tok, int tok_on_device, uint64_t salt,
+              uint64_t *keys_out, uint64_t *hit_bitmap_out, uint32_t *n_hit_chunks) {
+  return probe_impl(c, false, 0, tok, n_tok, tok_on_device, salt, keys_out, hit_bitmap_out,
+                    n_hit_chunks, nullptr);
+}
+
+int bsr_probe_request(bsr_ctx *c, uint64_t request_id, const int32_t *tok, size_t n_tok,
+                      int tok_on_device, uint64_t salt, uint64_t *keys_out, uint64_t *hit_bitmap_out,
+                      uint32_t *n_hit_chunks, int *tier_out) {
+  return probe_impl(c, true, request_id, tok, n_tok, tok_on_device, salt, keys_out, hit_bitmap_out,
+                    n_hit_chunks, tier_out);
+}
+
+int bsr_req_bind(bsr_ctx *c, bsr_req *q, uint64_t request_id, uint32_t tier) {
+  if (!c || !q || q->ctx != c || tier >= BSR_MAX_TIERS) return BSR_ERR_INVALID;
+  std::lock_guard<std::mutex> rl(c->restore_mu);
+  q->request_id = request_id;
+  q->tier = tier;
+  q->bound = true;
+  return BSR_OK;
+}
+
+int bsr_request_done(bsr_ctx *c, uint64_t request_id) {
+  if (!c) return BSR_ERR_INVALID;
+  std::lock_guard<std::mutex> lk(c->mu);
+  c->force_local.erase(request_id);
+  return BSR_OK;
+}
+
+int bsr_request_is_force_local(bsr_ctx *c, uint64_t request_id, int *out) {
+  if (!c || !out) return BSR_ERR_INVALID;
+  std::lock_guard<std::mutex> lk(c->mu);
+  *out = c->force_local.count(request_id) ? 1 : 0;
   return BSR_OK;
 }
 
@@ -1079,13 +1162,22 @@ int bsr_restore(bsr_ctx *c, bsr_req *q, void *cuda_stream) {
   clear_request_state(q);
   q->failed = false;
   const uint32_t R = c->cfg.n_ranks, N = q->n_adv;
+  uint64_t installed_before[BSR_MAX_RANKS];
+  for (uint32_t r = 0; r < BSR_MAX_RANKS; ++r) installed_before[r] = c->st.bytes_installed[r];
   if (N) {
     const size_t cells = (size_t)R * c->G * N;
     memset(q->h_ck, 0, cells * 8);
     memset(q->h_verdict, 0, cells * 4);
   }
   int rc = BSR_OK;
-  if (N) {
+  bool tier_up;
+  {
+    std::lock_guard<std::mutex> lk(c->mu);
+    tier_up = c->tier_available[q->tier];
+  }
+  if (!tier_up) {
+    rc = fail(c, BSR_ERR_TRANSFER, "tier %u is unavailable", q->tier);
+  } else if (N) {
     // are all advertised chunks already in device memory?  (then no staging is needed at all)
     std::vector<TierObj> objs((size_t)N * R);
     bool all_device = true;
@@ -1093,8 +1185,9 @@ int bsr_restore(bsr_ctx *c, bsr_req *q, void *cuda_stream) {
       std::lock_guard<std::mutex> lk(c->mu);
       for (uint32_t i = 0; i < N && all_device; ++i)
         for (uint32_t r = 0; r < R; ++r) {
-          auto it = c->tier[r].find(q->keys[i]);
-          if (it == c->tier[r].end() || it->second.loc != BSR_LOC_DEVICE) {
+          auto it = c->tier[q->tier][r].find(q->keys[i]);
+          if (!c->tier_available[q->tier] || it == c->tier[q->tier][r].end() ||
+              it->second.loc != BSR_LOC_DEVICE) {
             all_device = false;
             break;
           }
@@ -1116,10 +1209,16 @@ int bsr_restore(bsr_ctx *c, bsr_req *q, void *cuda_stream) {
         rc = fail(c, BSR_ERR_TIMEOUT, "a bounded wait inside the install kernel gave up");
     }
   }
-  if (rc == BSR_OK)
+  if (rc == BSR_OK) {
     q->restored = true;
-  else
+  } else {
     invalidate_host(q);
+    if (q->bound) {  // the next admission pass of this request must not re-enter the same fault
+      std::lock_guard<std::mutex> lk(c->mu);
+      c->force_local.insert(q->request_id);
+    }
+  }
+  for (uint32_t r = 0; r < R; ++r) c->st.bytes_restored_by_tier[q->tier] += c->st.bytes_installed[r] - installed_before[r];
   c->inject.kind = BSR_INJECT_NONE;  // one shot
   c->st.last_restore_ms = std::chrono::duration<double, std::milli>(Clock::now() - t0).count();
   return rc;
