@@ -301,7 +301,7 @@ def run_gpu(args):
     h2d_gbs = measure_h2d(torch, dev, chunk)
     e2e = Side(B, torch, dev, layout, R, N, W, payload, B.BSR_LOC_HOST,
                load_concurrency=args.load_concurrency, dev_staging_depth=args.depth,
-               install_variant=args.variant)
+               install_variant=args.variant, direct_install=args.direct)
     e2e.fill_tier(keys)
     e2e_steps = max(3, min(args.steps, 10))
     ms_e2e, st_e2e = timed_steps(torch, dist, world, e2e, tok, len(tok), salt, False, e2e_steps,
@@ -340,7 +340,8 @@ def run_gpu(args):
                    "rank_slices_per_gpu": R, "W": W,
                    "l2": "inputs (4.2 GB per step) are larger than L2; no flush needed",
                    "value_path": "tier resident in HBM, probe+restore+commit",
-                   "e2e_path": f"host tier -> pinned ring -> H2D -> install; load_concurrency="
+                   "e2e_path": ("host tier -> pinned ring -> install kernel reads the slots over the link; " if args.direct else
+                                "host tier -> pinned ring -> H2D -> install; ") + f"load_concurrency="
                                f"{args.load_concurrency}, dev_staging_depth={args.depth}"},
         "per_rank_GBps": value / (world * R),
         "restore_seconds": ms_res / 1e3,
@@ -420,6 +421,7 @@ def main():
     ap.add_argument("--depth", type=int, default=4)
     ap.add_argument("--variant", type=int, default=0, help="install kernel: 0 auto, 1 vector, 2 bulk copy")
     ap.add_argument("--chunks", type=int, default=0, help="prefix length in chunks (default: the workload's 128)")
+    ap.add_argument("--direct", action="store_true", help="e2e arm: staging-free install (kernel reads the pinned slots)")
     ap.add_argument("--sweep", action="store_true", help="e2e GB/s vs W and vs fill concurrency (long prefixes)")
     ap.add_argument("--resident-only", action="store_true", help="small profiling runs: skip e2e and CPU legs")
     args = ap.parse_args()

@@ -81,6 +81,11 @@ typedef struct bsr_config {
   uint32_t install_variant;   /* BSR_INSTALL_*                                                   */
   uint32_t time_kernels;      /* nonzero: bracket every install launch with CUDA events and
                                  accumulate bsr_stats.install_kernel_ms                          */
+  uint32_t direct_install;    /* nonzero: no device staging and no copy-engine transfer; the install
+                                 kernel reads the pinned slots over the host link itself (the
+                                 staging-free design point of the paper's "Avoiding staging"
+                                 discussion): HBM sees each payload byte once instead of three times */
+  uint32_t reserved;          /* must be 0                                                       */
 } bsr_config;
 
 typedef struct bsr_group_desc {

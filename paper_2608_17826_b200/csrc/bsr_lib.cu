@@ -116,6 +116,7 @@ struct bsr_ctx {
   // ring
   bool ring_ready = false;
   uint8_t *ring[BSR_MAX_RANKS] = {};
+  uint8_t *ring_dev[BSR_MAX_RANKS] = {};  // device-side addresses of the pinned rings
   uint8_t *dstage[BSR_MAX_RANKS] = {};
   std::vector<cudaEvent_t> ev_h2d, ev_inst, ev_start;  // [R*D]
   std::vector<std::pair<cudaEvent_t, cudaEvent_t>> ev_pool;  // launch timing, device-resident restores
@@ -237,8 +238,8 @@ uint32_t install_grid(const BsrInstallParams &p) {
   return (uint32_t)(total < want ? total : want);
 }
 
-int launch_install(bsr_ctx *c, const BsrInstallParams &p, cudaStream_t s) {
-  if (c->cfg.install_variant != BSR_INSTALL_VECTOR) {  // AUTO = bulk: the faster of the two on B200
+int launch_install(bsr_ctx *c, const BsrInstallParams &p, cudaStream_t s, bool host_source = false) {
+  if (c->cfg.install_variant != BSR_INSTALL_VECTOR && !host_source) {  // AUTO = bulk: the faster of the two on B200
     if (!c->bulk_ready) {
       CU(c, cudaFuncSetAttribute(bsr_install_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  BSR_K_BULK_SMEM));
@@ -364,13 +365,15 @@ int ensure_ring(bsr_ctx *c) {
   if (c->ring_ready) return BSR_OK;
   const uint32_t R = c->cfg.n_ranks, W = c->cfg.window_chunks, D = c->cfg.dev_staging_depth;
   for (uint32_t r = 0; r < R; ++r) {
-    if (cudaHostAlloc((void **)&c->ring[r], (size_t)W * c->slot_bytes, cudaHostAllocDefault) !=
-        cudaSuccess) {
+    if (cudaHostAlloc((void **)&c->ring[r], (size_t)W * c->slot_bytes, cudaHostAllocMapped) !=
+            cudaSuccess ||
+        cudaHostGetDevicePointer((void **)&c->ring_dev[r], c->ring[r], 0) != cudaSuccess) {
       cudaGetLastError();
       return fail(c, BSR_ERR_NOMEM, "pinned ring of %u x %llu bytes", W,
                   (unsigned long long)c->slot_bytes);
     }
     c->st.ring_bytes_allocated[r] = (uint64_t)W * c->slot_bytes;
+    if (c->cfg.direct_install) continue;  // no device staging: the kernel reads the slots itself
     if (cudaMalloc((void **)&c->dstage[r], (size_t)D * c->chunk_bytes) != cudaSuccess) {
       cudaGetLastError();
       return fail(c, BSR_ERR_NOMEM, "device staging of %u x %llu bytes", D,
@@ -506,6 +509,7 @@ int restore_ring(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_point 
   const uint32_t R = c->cfg.n_ranks, W = c->cfg.window_chunks, D = c->cfg.dev_staging_depth;
   const uint32_t N = q->n_adv, total = N * R;
   const uint32_t P = c->pieces;
+  const bool direct = c->cfg.direct_install != 0;
   std::vector<std::atomic<int>> state((size_t)total * P);  // per piece: 0 pending, 1 ready, <0 error
   for (auto &s : state) s.store(0, std::memory_order_relaxed);
   std::vector<TierObj> objs(total);
@@ -581,7 +585,7 @@ int restore_ring(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_point 
     // is complete, the install kernel on the compute stream
     while (!stop && submitted < admitted && submitted - reaped < R * D) {
       const uint32_t i = submitted / R, r = submitted % R, d = i % D, k = r * D + d;
-      uint8_t *stage = c->dstage[r] + (size_t)d * c->chunk_bytes;
+      uint8_t *stage = direct ? nullptr : c->dstage[r] + (size_t)d * c->chunk_bytes;
       cudaError_t e = cudaSuccess;
       bool blocked = false;
       while (cur_piece < P) {
@@ -600,23 +604,27 @@ int restore_ring(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_point 
         const uint8_t *from = (o.loc == BSR_LOC_HOST)
                                   ? c->ring[r] + (size_t)(i % W) * c->slot_bytes + off
                                   : o.data + off;
-        if (cur_piece == 0) e = cudaStreamWaitEvent(c->copy_stream, c->ev_inst[k], 0);
-        if (e == cudaSuccess)
-          e = cudaMemcpyAsync(stage + off, from, len, cudaMemcpyDefault, c->copy_stream);
-        if (e != cudaSuccess) {
-          first_error(fail(c, BSR_ERR_TRANSFER, "copy submit: %s", cudaGetErrorString(e)));
-          break;
+        if (!direct) {
+          if (cur_piece == 0) e = cudaStreamWaitEvent(c->copy_stream, c->ev_inst[k], 0);
+          if (e == cudaSuccess)
+            e = cudaMemcpyAsync(stage + off, from, len, cudaMemcpyDefault, c->copy_stream);
+          if (e != cudaSuccess) {
+            first_error(fail(c, BSR_ERR_TRANSFER, "copy submit: %s", cudaGetErrorString(e)));
+            break;
+          }
+          c->st.h2d_copies++;
         }
-        c->st.h2d_copies++;
         c->st.bytes_filled[r] += (o.loc == BSR_LOC_HOST) ? len : 0;
-        c->st.bytes_h2d[r] += len;
+        c->st.bytes_h2d[r] += len;  // bytes that cross the host link, by copy or by kernel loads
         ++cur_piece;
         progress = true;
       }
       if (stop || blocked) break;
       const TierObj &o = objs[submitted];
-      e = cudaEventRecord(c->ev_h2d[k], c->copy_stream);
-      if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, c->ev_h2d[k], 0);
+      if (!direct) {
+        e = cudaEventRecord(c->ev_h2d[k], c->copy_stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, c->ev_h2d[k], 0);
+      }
       if (e == cudaSuccess && c->cfg.time_kernels) e = cudaEventRecord(c->ev_start[k], stream);
       if (e != cudaSuccess) {
         first_error(fail(c, BSR_ERR_TRANSFER, "copy submit: %s", cudaGetErrorString(e)));
@@ -630,11 +638,14 @@ int restore_ring(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_point 
       p.ck_out = q->d_ck;
       p.verdict = q->d_verdict;
       p.n_chunks = 1;
-      p.one.src = stage;
+      // direct mode: the kernel reads the pinned slot (or the device object) itself over the link
+      p.one.src = !direct ? stage
+                          : (o.loc == BSR_LOC_HOST ? c->ring_dev[r] + (size_t)(i % W) * c->slot_bytes
+                                                   : o.data);
       p.one.chunk = i;
       p.one.rank = r;
       for (uint32_t g = 0; g < c->G; ++g) p.one.expect[g] = o.ck[g];
-      const int lrc = launch_install(c, p, stream);
+      const int lrc = launch_install(c, p, stream, direct && o.loc == BSR_LOC_HOST);
       e = cudaEventRecord(c->ev_inst[k], stream);
       if (lrc != BSR_OK || e != cudaSuccess) {
         first_error(lrc != BSR_OK ? lrc : fail(c, BSR_ERR_CUDA, "record: %s", cudaGetErrorString(e)));

@@ -288,3 +288,24 @@ def test_bulk_install_kernel_detects_corruption_and_computes_store_checksums():
         case.payload[(1, 3)][lo:hi].view("<u4")[12345] ^= np.uint32(0x10)
         assert gpu.restore() == B.BSR_ERR_CHECKSUM
         assert gpu.commit() == 0 and (gpu.bitmap(4) == 0).all()
+
+
+# ---------------------------------------------------------------- staging-free (direct) install
+@pytest.mark.parametrize("layout_name,R,N,W", [("tiny", 2, 23, 4), ("hetero", 2, 6, 4), ("baseline", 2, 10, 4)])
+def test_direct_install_from_pinned_slots_matches_oracle(layout_name, R, N, W):
+    layout = {"tiny": synth.tiny_layout, "hetero": synth.hetero_layout,
+              "baseline": synth.baseline_layout}[layout_name]()
+    case = Case(layout, R, N, seed=1000 + N)
+    ora = run_oracle(case, W)
+    with GpuSide(case, W, direct_install=True) as gpu:
+        rc, keys, bm, n_hit = gpu.probe()
+        gpu.request(keys, n_hit)
+        assert gpu.restore() == gpu.B.BSR_OK, gpu.B.bsr_last_error(gpu.ctx)
+        _check_success(case, W, gpu, ora, N)
+        st = gpu.stats()
+        assert st.h2d_copies == 0                                  # nothing went through the copy engine
+        # corruption in a slot is still caught, exposure still collapses
+        r, g, i, frac = synth.fault_site(R, case.G, 1, N, case=11, seed=3)
+        gpu.B.bsr_test_inject(gpu.ctx, gpu.B.BSR_INJECT_CORRUPT_SLOT, r, g, i, frac)
+        assert gpu.restore() == gpu.B.BSR_ERR_CHECKSUM
+        assert gpu.commit() == 0 and (gpu.bitmap(N) == 0).all()

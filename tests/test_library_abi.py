@@ -33,7 +33,7 @@ def test_binding_covers_the_header_and_struct_sizes_match():
     assert sorted(B.EXPORTS) == _declared()
     for n in B.EXPORTS:
         assert callable(getattr(B, n))
-    assert ctypes.sizeof(B.bsr_config) == 48  # as gcc lays out include/bsr.h
+    assert ctypes.sizeof(B.bsr_config) == 56  # as gcc lays out include/bsr.h
     assert ctypes.sizeof(B.bsr_tensor_desc) == 16
     assert ctypes.sizeof(B.bsr_stats) == 8 * 8 * 5 + 8 * 7 + 8 * 4 + 8 * 2
 
