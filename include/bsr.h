@@ -85,7 +85,11 @@ typedef struct bsr_config {
                                  kernel reads the pinned slots over the host link itself (the
                                  staging-free design point of the paper's "Avoiding staging"
                                  discussion): HBM sees each payload byte once instead of three times */
-  uint32_t reserved;          /* must be 0                                                       */
+  uint32_t budget_slots;      /* 0: restores on this context are serialised by a lock and each owns W
+                                 slots per rank (the paper's prototype).  B > 0: a global admission
+                                 budget (Section 7 "Current concurrency is conservative"): restores
+                                 run concurrently and share a pool of B slots per rank; each holds
+                                 at most W, together never more than B                            */
 } bsr_config;
 
 typedef struct bsr_group_desc {

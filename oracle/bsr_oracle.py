@@ -405,3 +405,69 @@ def restore_request(eng: Engine, request_id: int, tier: int, reg: Registration, 
 def request_done(eng: Engine, request_id: int):
     """Successful RUNNING admission or request teardown removes the marker."""
     eng.force_local.discard(request_id)
+
+
+# --------------------------------------------------------------------------------------
+# several restores under one admission budget  (Section 7 "Current concurrency is
+# conservative": allow several request windows whenever their aggregate RWS stays below B)
+# --------------------------------------------------------------------------------------
+def restore_concurrent(reg: Registration, tiers: list[Tier], reqs: list[Request],
+                       paged: list[list[np.ndarray]], W: int, B: int):
+    """Restores several requests into the same paged pools under a budget of B staging slots per
+    rank.  The model is synchronous rounds: in every round each unfinished request, in order,
+    admits its next window of min(W, chunks left, slots still free in the budget) chunks; all
+    admitted windows are fetched, verified and installed as in `restore`; then all are released.
+    Every request keeps Eq. 3 (at most W live), all together never exceed B.  A failing request is
+    invalidated alone: the others' outcomes do not depend on it.
+    Returns (status per request, peak aggregate staging bytes per rank, rounds)."""
+    R = reqs[0].n_ranks
+    Q = len(reqs)
+    done = [0] * Q
+    status = [OK] * Q
+    for q in reqs:
+        q.valid[:] = False
+        q.restored, q.failed = False, False
+    peak = [0] * R
+    rounds = 0
+    while any(status[k] == OK and done[k] < reqs[k].n_adv for k in range(Q)):
+        rounds += 1
+        free = B
+        windows = []
+        for k in range(Q):
+            if status[k] != OK or done[k] >= reqs[k].n_adv:
+                continue
+            w = min(W, reqs[k].n_adv - done[k], free)
+            if w <= 0:
+                continue
+            free -= w
+            windows.append((k, range(done[k], done[k] + w)))
+        live = sum(len(win) for _, win in windows) * reg.slot_bytes
+        for r in range(R):
+            peak[r] = max(peak[r], live)
+        for k, win in windows:
+            q = reqs[k]
+            for r in range(R):
+                for i in win:
+                    obj = tiers[r].get(q.keys[i])
+                    if obj is None:
+                        status[k] = ERR_MISSING
+                        break
+                    data, cks = obj[0].copy(), obj[1]
+                    for g in range(reg.n_groups):
+                        if checksum(data[slice(*reg.segment(g))]) != cks[g]:
+                            status[k] = ERR_CHECKSUM
+                            break
+                        scatter_chunk_group(reg, g, data, i, q.block_tables[r][g], paged[r])
+                        q.valid[r, g, i] = True
+                    if status[k] != OK:
+                        break
+                if status[k] != OK:
+                    break
+            if status[k] != OK:
+                invalidate(reg, q, paged, scrub=False)
+            else:
+                done[k] += len(win)
+    for k in range(Q):
+        if status[k] == OK:
+            reqs[k].restored = True
+    return status, peak, rounds

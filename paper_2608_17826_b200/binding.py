@@ -43,7 +43,7 @@ class bsr_config(C.Structure):
                 ("load_concurrency", C.c_uint32), ("dev_staging_depth", C.c_uint32),
                 ("timeout_ms", C.c_uint32), ("slot_align", C.c_uint32), ("device", C.c_int32),
                 ("reg_id", C.c_uint64), ("install_variant", C.c_uint32), ("time_kernels", C.c_uint32),
-                ("direct_install", C.c_uint32), ("reserved", C.c_uint32)]
+                ("direct_install", C.c_uint32), ("budget_slots", C.c_uint32)]
 
 
 class bsr_group_desc(C.Structure):
@@ -128,10 +128,10 @@ def _ptr(a) -> int | None:
 def bsr_ctx_create(W: int, n_ranks: int, *, load_concurrency: int = 0, dev_staging_depth: int = 0,
                    timeout_ms: int = 0, slot_align: int = 0, device: int = 0, reg_id: int = 1,
                    install_variant: int = BSR_INSTALL_AUTO, time_kernels: bool = False,
-                   direct_install: bool = False):
+                   direct_install: bool = False, budget_slots: int = 0):
     cfg = bsr_config(W, n_ranks, BSR_CHUNK_TOKENS, load_concurrency, dev_staging_depth, timeout_ms,
                      slot_align, device, reg_id, install_variant, int(time_kernels),
-                     int(direct_install), 0)
+                     int(direct_install), budget_slots)
     ctx = C.c_void_p()
     rc = lib.bsr_ctx_create(C.byref(cfg), C.byref(ctx))
     return rc, (ctx if rc == BSR_OK else None)

@@ -1,6 +1,15 @@
 // Host side of the BSR library: context, registration, chunk index, probe, the W-slot window
-// pipeline (pinned ring -> copy stream -> device staging -> install kernel), commit, invalidate.
-// The C interface is declared in include/bsr.h.
+// pipeline (pinned slot pool -> copy stream -> device staging -> install kernel), commit,
+// invalidate, request-level recovery.  The C interface is declared in include/bsr.h.
+//
+// Locks (never nested among the short ones, listed outermost first):
+//   req->mu      one call at a time per request object (restore holds it for its whole duration)
+//   restore_mu   the paper's bounded-retrieve lock: held by a whole restore unless an admission
+//                budget is configured, in which case restores run concurrently and share B slots
+//   aux_mu       probe, store-path checksums and scrub: they share context-level scratch and a stream
+//   setup_mu     one-time set-up: tile table, slot pool, per-restore device resources
+//   fill_mu      the fill task queue;  pool_mu  the slot pool and live/peak accounting
+//   mu           tier index, statistics, force-local markers, error text
 #include "../../include/bsr.h"
 
 #include <immintrin.h>
@@ -11,6 +20,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <memory>
 #include <mutex>
 #include <new>
 #include <string>
@@ -27,7 +37,7 @@ using Clock = std::chrono::steady_clock;
 
 constexpr int kInstallThreads = 256;
 constexpr int kInstallUnroll = 4;
-constexpr int kLaunchSlots = 8;  // independent scratch sets for install launches in flight
+constexpr int kLaunchSlots = 8;  // scratch sets for batched install launches in flight per restore
 constexpr uint32_t kSmCount = 148;
 constexpr uint64_t kPieceBytes = 8ull << 20;  // fill and host-to-device copy granularity
 
@@ -50,10 +60,44 @@ struct Inject {
   uint64_t seed = 0;
 };
 
+// Device-side resources of one restore in flight.  Pooled: a finished restore hands them back.
+struct JobRes {
+  cudaStream_t stream = nullptr;                        // used when the caller passes no stream
+  uint8_t *dstage[BSR_MAX_RANKS] = {};                  // D staging buffers per rank
+  std::vector<cudaEvent_t> ev_h2d, ev_inst, ev_start;   // [R*D]
+  std::vector<std::pair<cudaEvent_t, cudaEvent_t>> ev_pool;  // launch timing, batched launches
+  cudaEvent_t ev_done = nullptr;
+  uint64_t *d_acc = nullptr;      // [n_slots][BATCH][GROUPS] checksum accumulators, kept zero
+  unsigned int *d_cnt = nullptr;  // [n_slots] CTA counters, kept zero; [n_slots] = error flag
+  uint32_t n_slots = 0;
+  uint64_t seq = 0;
+};
+
+// Counters a restore accumulates privately and merges into the context statistics at its end.
+struct StatDelta {
+  uint64_t bytes_filled[BSR_MAX_RANKS] = {}, bytes_h2d[BSR_MAX_RANKS] = {},
+           bytes_installed[BSR_MAX_RANKS] = {};
+  uint64_t windows = 0, kernel_launches = 0, h2d_copies = 0, install_launches = 0;
+  double install_kernel_ms = 0.0;
+};
+
+// Host-side state of one restore through the slot pool.
+struct Job {
+  bsr_req *q = nullptr;
+  Clock::time_point deadline;
+  uint32_t P = 1;
+  std::unique_ptr<std::atomic<int>[]> state;  // per piece: 0 pending, 1 ready, <0 error
+  std::vector<TierObj> objs;                  // per (chunk, rank)
+  std::vector<uint32_t> slot;                 // per (chunk, rank): slot of the rank's pool
+  std::atomic<bool> abort{false};
+  uint32_t fill_admitted = 0, fill_next = 0, fill_active = 0;  // guarded by fill_mu
+};
+
 }  // namespace
 
 struct bsr_req {
   bsr_ctx *ctx = nullptr;
+  std::mutex mu;
   uint32_t n_adv = 0;
   std::vector<uint64_t> keys;
   std::vector<std::vector<int32_t>> tables;  // [R*G]
@@ -76,8 +120,8 @@ struct bsr_req {
 
 struct bsr_ctx {
   bsr_config cfg{};
-  std::mutex mu;          // registration, tier index, stats, error text
-  std::mutex restore_mu;  // one bounded restore at a time
+  uint32_t budget = 0;  // B: slots per rank shared by all restores (= W without an admission budget)
+  std::mutex mu, restore_mu, aux_mu, setup_mu, fill_mu, pool_mu;
   std::string err;
 
   // registration
@@ -87,59 +131,45 @@ struct bsr_ctx {
   std::vector<TensorReg> tensors;
   uint64_t chunk_bytes = 0, slot_bytes = 0;
   uint64_t seg_begin[BSR_MAX_GROUPS] = {}, seg_bytes[BSR_MAX_GROUPS] = {};
-  bool finalized = false;
+  uint32_t pieces = 1;  // fill pieces per chunk
+  std::atomic<bool> finalized{false};
   std::vector<BsrTile> h_tiles;
   BsrTile *d_tiles = nullptr;
   uint64_t *d_tensor_base = nullptr;
   uint32_t *d_tensor_group = nullptr, *d_tensor_run = nullptr;
 
-  // tier + index
+  // tiers + index (mu)
   std::unordered_map<uint64_t, TierObj> tier[BSR_MAX_TIERS][BSR_MAX_RANKS];
   bool tier_available[BSR_MAX_TIERS] = {true, true, true, true};
   std::unordered_set<uint64_t> force_local;  // request ids whose next probe must report zero
+  Inject inject;
+  bsr_stats st{};
+
+  // context-level stream and scratch for probe, store-path checksums, scrub (aux_mu)
+  cudaStream_t copy_stream = nullptr, own_stream = nullptr;
+  JobRes aux;
   uint8_t *d_put_stage = nullptr;
   uint64_t *h_put_ck = nullptr, *d_put_ck = nullptr;  // pinned [G] sums + verdict dump
   uint32_t *h_put_verdict = nullptr, *d_put_verdict = nullptr;
-
-  // streams and scratch
-  cudaStream_t copy_stream = nullptr, own_stream = nullptr;
-  uint64_t *d_acc = nullptr;        // [kLaunchSlots][BATCH][GROUPS]
-  unsigned int *d_counters = nullptr;  // [kLaunchSlots] install + [1] probe + [1] err flag
-  uint64_t launch_seq = 0;
-  bool bulk_ready = false;  // dynamic shared memory limit of the bulk kernel has been raised
-
-  // probe scratch (grown on demand)
+  unsigned int *d_probe_cnt = nullptr;
   int32_t *d_tok = nullptr;
   uint64_t *d_digests = nullptr, *d_keys = nullptr, *h_keys = nullptr;
   size_t probe_cap_chunks = 0;
 
-  // ring
-  bool ring_ready = false;
+  // slot pool (setup_mu to create, pool_mu to use)
+  std::atomic<bool> ring_ready{false};
   uint8_t *ring[BSR_MAX_RANKS] = {};
   uint8_t *ring_dev[BSR_MAX_RANKS] = {};  // device-side addresses of the pinned rings
-  uint8_t *dstage[BSR_MAX_RANKS] = {};
-  std::vector<cudaEvent_t> ev_h2d, ev_inst, ev_start;  // [R*D]
-  std::vector<std::pair<cudaEvent_t, cudaEvent_t>> ev_pool;  // launch timing, device-resident restores
-  cudaEvent_t ev_done = nullptr;
+  std::vector<uint32_t> free_slots[BSR_MAX_RANKS];
+  uint64_t live_total[BSR_MAX_RANKS] = {};
+  std::vector<JobRes *> res_free, res_all;  // setup_mu
 
-  // filler pool
+  // fill task queue (fill_mu)
   std::vector<std::thread> fillers;
-  std::mutex fill_mu;
   std::condition_variable fill_cv;
   bool fill_shutdown = false;
-  // state of the restore in progress, guarded by fill_mu unless atomic
-  bsr_req *cur_req = nullptr;
-  uint32_t fill_total = 0, fill_admitted = 0, fill_next = 0;
-  std::atomic<bool> fill_abort{false};
-  Clock::time_point fill_deadline;
-  std::vector<std::atomic<int>> *task_state = nullptr;  // 0 pending, 1 ready, <0 error
-  std::vector<TierObj> *task_obj = nullptr;
-  uint32_t fill_active = 0;
-  uint32_t pieces = 1;  // fill pieces per chunk
-
-  Inject inject;
-  bsr_stats st{};
-  uint64_t live[BSR_MAX_RANKS] = {};
+  std::vector<Job *> jobs;
+  size_t rr = 0;
 };
 
 namespace {
@@ -167,9 +197,23 @@ int fail(bsr_ctx *c, int code, const char *fmt, ...) {
 
 uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 
-// ---- registration -> tile table ----------------------------------------------------------------
+void merge_stats(bsr_ctx *c, const StatDelta &d) {
+  std::lock_guard<std::mutex> g(c->mu);
+  for (uint32_t r = 0; r < BSR_MAX_RANKS; ++r) {
+    c->st.bytes_filled[r] += d.bytes_filled[r];
+    c->st.bytes_h2d[r] += d.bytes_h2d[r];
+    c->st.bytes_installed[r] += d.bytes_installed[r];
+  }
+  c->st.windows += d.windows;
+  c->st.kernel_launches += d.kernel_launches;
+  c->st.h2d_copies += d.h2d_copies;
+  c->st.install_launches += d.install_launches;
+  c->st.install_kernel_ms += d.install_kernel_ms;
+}
+
+// ---- registration -> tile table (setup_mu held) --------------------------------------------------
 int finalize_registration(bsr_ctx *c) {
-  if (c->finalized) return BSR_OK;
+  if (c->finalized.load(std::memory_order_acquire)) return BSR_OK;
   if (c->L == 0) return fail(c, BSR_ERR_STATE, "no registration");
   for (uint32_t r = 0; r < c->cfg.n_ranks; ++r)
     if (!c->rank_registered[r]) return fail(c, BSR_ERR_STATE, "rank %u is not registered", r);
@@ -214,12 +258,23 @@ int finalize_registration(bsr_ctx *c) {
   CU(c, cudaMemcpy(c->d_tensor_group, tgroup.data(), c->L * 4, cudaMemcpyHostToDevice));
   CU(c, cudaMalloc(&c->d_tensor_run, c->L * 4));
   CU(c, cudaMemcpy(c->d_tensor_run, trun.data(), c->L * 4, cudaMemcpyHostToDevice));
-  c->st.dev_aux_bytes += c->h_tiles.size() * sizeof(BsrTile) + bases.size() * 8 + c->L * 8;
-  c->finalized = true;
+  CU(c, cudaFuncSetAttribute(bsr_install_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             BSR_K_BULK_SMEM));
+  {
+    std::lock_guard<std::mutex> g(c->mu);
+    c->st.dev_aux_bytes += c->h_tiles.size() * sizeof(BsrTile) + bases.size() * 8 + c->L * 8;
+  }
+  c->finalized.store(true, std::memory_order_release);
   return BSR_OK;
 }
 
-void fill_params(bsr_ctx *c, BsrInstallParams &p, uint32_t slot) {
+int ensure_finalized(bsr_ctx *c) {
+  if (c->finalized.load(std::memory_order_acquire)) return BSR_OK;
+  std::lock_guard<std::mutex> sl(c->setup_mu);
+  return finalize_registration(c);
+}
+
+void fill_params(bsr_ctx *c, BsrInstallParams &p, JobRes *res, uint32_t slot) {
   p.tiles = c->d_tiles;
   p.n_tiles = (uint32_t)c->h_tiles.size();
   p.n_groups = c->G;
@@ -227,36 +282,102 @@ void fill_params(bsr_ctx *c, BsrInstallParams &p, uint32_t slot) {
   p.tensor_base = c->d_tensor_base;
   for (uint32_t g = 0; g < c->G; ++g)
     p.blocks_per_chunk[g] = BSR_CHUNK_TOKENS / c->groups[g].block_tokens;
-  p.acc = c->d_acc + (size_t)slot * BSR_K_MAX_BATCH * BSR_K_MAX_GROUPS;
-  p.ctas_done = c->d_counters + slot;
-  p.err_flag = c->d_counters + kLaunchSlots + 1;
+  p.acc = res->d_acc + (size_t)slot * BSR_K_MAX_BATCH * BSR_K_MAX_GROUPS;
+  p.ctas_done = res->d_cnt + slot;
+  p.err_flag = res->d_cnt + res->n_slots;
 }
 
-uint32_t install_grid(const BsrInstallParams &p) {
+// host_source: the chunk is read from mapped host memory; plain loads are used for that.
+int launch_install(bsr_ctx *c, const BsrInstallParams &p, cudaStream_t s, StatDelta &sd,
+                   bool host_source = false) {
   const uint64_t total = (uint64_t)p.n_chunks * p.n_tiles;
-  const uint64_t want = (uint64_t)kSmCount * 8;
-  return (uint32_t)(total < want ? total : want);
-}
-
-int launch_install(bsr_ctx *c, const BsrInstallParams &p, cudaStream_t s, bool host_source = false) {
-  if (c->cfg.install_variant != BSR_INSTALL_VECTOR && !host_source) {  // AUTO = bulk: the faster of the two on B200
-    if (!c->bulk_ready) {
-      CU(c, cudaFuncSetAttribute(bsr_install_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 BSR_K_BULK_SMEM));
-      c->bulk_ready = true;
-    }
-    const uint64_t total = (uint64_t)p.n_chunks * p.n_tiles;
+  if (c->cfg.install_variant != BSR_INSTALL_VECTOR && !host_source) {  // AUTO = bulk copies
     const uint64_t want = (uint64_t)kSmCount * 2;  // two CTAs of 6 x 16 KiB stages per SM
-    const uint32_t grid = (uint32_t)(total < want ? total : want);
-    bsr_install_bulk_kernel<<<grid, BSR_K_BULK_THREADS, BSR_K_BULK_SMEM, s>>>(p);
+    bsr_install_bulk_kernel<<<(uint32_t)(total < want ? total : want), BSR_K_BULK_THREADS,
+                              BSR_K_BULK_SMEM, s>>>(p);
   } else {
+    const uint64_t want = (uint64_t)kSmCount * 8;
     bsr_install_vec_kernel<kInstallThreads, kInstallUnroll>
-        <<<install_grid(p), kInstallThreads, 0, s>>>(p);
+        <<<(uint32_t)(total < want ? total : want), kInstallThreads, 0, s>>>(p);
   }
   CU(c, cudaGetLastError());
-  c->st.kernel_launches++;
-  c->st.install_launches++;
+  sd.kernel_launches++;
+  sd.install_launches++;
   return BSR_OK;
+}
+
+// ---- per-restore device resources ----------------------------------------------------------------
+void destroy_res(JobRes *res) {
+  for (uint32_t r = 0; r < BSR_MAX_RANKS; ++r)
+    if (res->dstage[r]) cudaFree(res->dstage[r]);
+  for (auto e : res->ev_h2d) cudaEventDestroy(e);
+  for (auto e : res->ev_inst) cudaEventDestroy(e);
+  for (auto e : res->ev_start) cudaEventDestroy(e);
+  for (auto &pr : res->ev_pool) {
+    cudaEventDestroy(pr.first);
+    cudaEventDestroy(pr.second);
+  }
+  if (res->ev_done) cudaEventDestroy(res->ev_done);
+  cudaFree(res->d_acc);
+  cudaFree(res->d_cnt);
+  if (res->stream) cudaStreamDestroy(res->stream);
+}
+
+int init_scratch(bsr_ctx *c, JobRes *res, uint32_t n_slots) {
+  res->n_slots = n_slots;
+  const size_t acc_bytes = (size_t)n_slots * BSR_K_MAX_BATCH * BSR_K_MAX_GROUPS * 8;
+  const size_t cnt_bytes = (n_slots + 1) * sizeof(unsigned int);
+  CU(c, cudaMalloc(&res->d_acc, acc_bytes));
+  CU(c, cudaMalloc(&res->d_cnt, cnt_bytes));
+  CU(c, cudaMemset(res->d_acc, 0, acc_bytes));
+  CU(c, cudaMemset(res->d_cnt, 0, cnt_bytes));
+  CU(c, cudaEventCreateWithFlags(&res->ev_done, cudaEventDisableTiming));
+  std::lock_guard<std::mutex> g(c->mu);
+  c->st.dev_aux_bytes += acc_bytes + cnt_bytes;
+  return BSR_OK;
+}
+
+// A resource set from the pool, or a new one (setup_mu taken here).
+int acquire_res(bsr_ctx *c, JobRes **out) {
+  std::lock_guard<std::mutex> sl(c->setup_mu);
+  if (!c->res_free.empty()) {
+    *out = c->res_free.back();
+    c->res_free.pop_back();
+    return BSR_OK;
+  }
+  const uint32_t R = c->cfg.n_ranks, D = c->cfg.dev_staging_depth;
+  JobRes *res = new (std::nothrow) JobRes();
+  if (!res) return BSR_ERR_NOMEM;
+  c->res_all.push_back(res);
+  CU(c, cudaStreamCreateWithFlags(&res->stream, cudaStreamNonBlocking));
+  int rc = init_scratch(c, res, R * D + kLaunchSlots);
+  if (rc != BSR_OK) return rc;
+  if (!c->cfg.direct_install) {
+    for (uint32_t r = 0; r < R; ++r) {
+      if (cudaMalloc((void **)&res->dstage[r], (size_t)D * c->chunk_bytes) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(c, BSR_ERR_NOMEM, "device staging of %u x %llu bytes", D,
+                    (unsigned long long)c->chunk_bytes);
+      }
+    }
+    std::lock_guard<std::mutex> g(c->mu);
+    c->st.dev_aux_bytes += (uint64_t)R * D * c->chunk_bytes;
+  }
+  res->ev_h2d.resize(R * D);
+  res->ev_inst.resize(R * D);
+  res->ev_start.resize(R * D);
+  for (uint32_t k = 0; k < R * D; ++k) {
+    CU(c, cudaEventCreateWithFlags(&res->ev_h2d[k], cudaEventDisableTiming));
+    CU(c, cudaEventCreate(&res->ev_inst[k]));
+    CU(c, cudaEventCreate(&res->ev_start[k]));
+  }
+  *out = res;
+  return BSR_OK;
+}
+
+void release_res(bsr_ctx *c, JobRes *res) {
+  std::lock_guard<std::mutex> sl(c->setup_mu);
+  c->res_free.push_back(res);
 }
 
 // ---- filler threads: tier object -> pinned slot -------------------------------------------------
@@ -291,32 +412,45 @@ void fill_copy(uint8_t *dst, const uint8_t *src, size_t n) {
     memcpy(dst, src, n);
 }
 
-// One fill task = one piece (at most kPieceBytes) of one chunk of one rank.  Pieces let the first
-// device copy start after a fraction of a chunk has been fetched and keep all threads busy on the
-// chunks the copy engine needs next.
+// One fill task = one piece (at most kPieceBytes) of one chunk of one rank of one restore.  Pieces
+// let the first device copy start after a fraction of a chunk has been fetched and keep all threads
+// busy on the chunks the copy engine needs next.  Restores in flight are served round-robin.
 void filler_main(bsr_ctx *c) {
   for (;;) {
-    uint32_t t;
-    bsr_req *req;
+    Job *job = nullptr;
+    uint32_t t = 0;
     {
       std::unique_lock<std::mutex> lk(c->fill_mu);
       c->fill_cv.wait(lk, [&] {
-        return c->fill_shutdown || (c->cur_req && c->fill_next < c->fill_admitted);
+        if (c->fill_shutdown) return true;
+        for (Job *j : c->jobs)
+          if (j->fill_next < j->fill_admitted) return true;
+        return false;
       });
       if (c->fill_shutdown) return;
-      t = c->fill_next++;
-      req = c->cur_req;
-      c->fill_active++;
+      const size_t n = c->jobs.size();
+      for (size_t k = 0; k < n; ++k) {
+        Job *j = c->jobs[(c->rr + k) % n];
+        if (j->fill_next < j->fill_admitted) {
+          job = j;
+          c->rr = (c->rr + k + 1) % n;
+          break;
+        }
+      }
+      t = job->fill_next++;
+      job->fill_active++;
     }
-    const uint32_t R = c->cfg.n_ranks, W = c->cfg.window_chunks, P = c->pieces;
+    bsr_req *req = job->q;
+    const uint32_t R = c->cfg.n_ranks, P = job->P;
     const uint32_t s = t / P, piece = t % P;
     const uint32_t i = s / R, r = s % R;
     const uint64_t off = (uint64_t)piece * kPieceBytes;
     const uint64_t len = (c->chunk_bytes - off < kPieceBytes) ? c->chunk_bytes - off : kPieceBytes;
     int state = 1;
     TierObj obj{};
-    if (!c->fill_abort.load(std::memory_order_acquire)) {
+    if (!job->abort.load(std::memory_order_acquire)) {
       bool found = false, tier_down = false;
+      Inject inj;
       {
         std::lock_guard<std::mutex> g(c->mu);
         auto &index = c->tier[req->tier][r];
@@ -326,8 +460,8 @@ void filler_main(bsr_ctx *c) {
           found = true;
         }
         if (!c->tier_available[req->tier]) tier_down = true;
+        inj = c->inject;
       }
-      const Inject inj = c->inject;
       const bool hit = inj.kind != BSR_INJECT_NONE && inj.rank == r && inj.chunk == i;
       if (tier_down) {
         state = BSR_ERR_TRANSFER;  // the tier went away after the probe
@@ -336,12 +470,12 @@ void filler_main(bsr_ctx *c) {
       } else if (hit && inj.kind == BSR_INJECT_FILL_ERROR) {
         state = BSR_ERR_TRANSFER;
       } else if (hit && inj.kind == BSR_INJECT_FILL_STALL && piece == 0) {
-        while (!c->fill_abort.load(std::memory_order_acquire) &&
-               Clock::now() < c->fill_deadline + std::chrono::seconds(5))
+        while (!job->abort.load(std::memory_order_acquire) &&
+               Clock::now() < job->deadline + std::chrono::seconds(5))
           std::this_thread::sleep_for(std::chrono::milliseconds(1));
         state = BSR_ERR_TIMEOUT;
       } else if (obj.loc == BSR_LOC_HOST) {
-        uint8_t *slot = c->ring[r] + (size_t)(i % W) * c->slot_bytes;
+        uint8_t *slot = c->ring[r] + (size_t)job->slot[s] * c->slot_bytes;
         fill_copy(slot + off, obj.data + off, len);
         if (hit && inj.kind == BSR_INJECT_CORRUPT_SLOT && inj.group < c->G) {
           const uint64_t words = c->seg_bytes[inj.group] / 4;
@@ -351,52 +485,41 @@ void filler_main(bsr_ctx *c) {
         }
       }
     }
-    if (piece == 0) (*c->task_obj)[s] = obj;
-    (*c->task_state)[t].store(state, std::memory_order_release);
+    if (piece == 0) job->objs[s] = obj;
+    job->state[t].store(state, std::memory_order_release);
     {
       std::lock_guard<std::mutex> lk(c->fill_mu);
-      c->fill_active--;
+      job->fill_active--;
     }
     c->fill_cv.notify_all();
   }
 }
 
+// The pinned slot pool: B slots per rank (B = W unless an admission budget is configured).
 int ensure_ring(bsr_ctx *c) {
-  if (c->ring_ready) return BSR_OK;
-  const uint32_t R = c->cfg.n_ranks, W = c->cfg.window_chunks, D = c->cfg.dev_staging_depth;
+  if (c->ring_ready.load(std::memory_order_acquire)) return BSR_OK;
+  std::lock_guard<std::mutex> sl(c->setup_mu);
+  if (c->ring_ready.load(std::memory_order_acquire)) return BSR_OK;
+  const uint32_t R = c->cfg.n_ranks, B = c->budget;
   for (uint32_t r = 0; r < R; ++r) {
-    if (cudaHostAlloc((void **)&c->ring[r], (size_t)W * c->slot_bytes, cudaHostAllocMapped) !=
+    if (cudaHostAlloc((void **)&c->ring[r], (size_t)B * c->slot_bytes, cudaHostAllocMapped) !=
             cudaSuccess ||
         cudaHostGetDevicePointer((void **)&c->ring_dev[r], c->ring[r], 0) != cudaSuccess) {
       cudaGetLastError();
-      return fail(c, BSR_ERR_NOMEM, "pinned ring of %u x %llu bytes", W,
+      return fail(c, BSR_ERR_NOMEM, "pinned pool of %u x %llu bytes", B,
                   (unsigned long long)c->slot_bytes);
     }
-    c->st.ring_bytes_allocated[r] = (uint64_t)W * c->slot_bytes;
-    if (c->cfg.direct_install) continue;  // no device staging: the kernel reads the slots itself
-    if (cudaMalloc((void **)&c->dstage[r], (size_t)D * c->chunk_bytes) != cudaSuccess) {
-      cudaGetLastError();
-      return fail(c, BSR_ERR_NOMEM, "device staging of %u x %llu bytes", D,
-                  (unsigned long long)c->chunk_bytes);
+    {
+      std::lock_guard<std::mutex> g(c->mu);
+      c->st.ring_bytes_allocated[r] = (uint64_t)B * c->slot_bytes;
     }
-    c->st.dev_aux_bytes += (uint64_t)D * c->chunk_bytes;
-  }
-  c->ev_h2d.resize(R * D);
-  c->ev_inst.resize(R * D);
-  c->ev_start.resize(R * D);
-  for (uint32_t k = 0; k < R * D; ++k) {
-    CU(c, cudaEventCreateWithFlags(&c->ev_h2d[k], cudaEventDisableTiming));
-    CU(c, cudaEventCreate(&c->ev_inst[k]));
-    CU(c, cudaEventCreate(&c->ev_start[k]));
+    std::lock_guard<std::mutex> pl(c->pool_mu);
+    c->free_slots[r].clear();
+    for (uint32_t k = B; k > 0; --k) c->free_slots[r].push_back(k - 1);
   }
   for (uint32_t k = 0; k < c->cfg.load_concurrency; ++k) c->fillers.emplace_back(filler_main, c);
-  c->ring_ready = true;
+  c->ring_ready.store(true, std::memory_order_release);
   return BSR_OK;
-}
-
-void clear_request_state(bsr_req *q) {
-  std::fill(q->bitmap.begin(), q->bitmap.end(), 0ull);
-  q->restored = false;
 }
 
 void invalidate_host(bsr_req *q) {
@@ -405,7 +528,7 @@ void invalidate_host(bsr_req *q) {
 }
 
 // Reads the verdicts of chunk i of rank r after its install event completed.
-int harvest(bsr_ctx *c, bsr_req *q, uint32_t r, uint32_t i) {
+int harvest(bsr_ctx *c, bsr_req *q, uint32_t r, uint32_t i, StatDelta &sd) {
   int rc = BSR_OK;
   for (uint32_t g = 0; g < c->G; ++g) {
     const size_t o = ((size_t)r * c->G + g) * q->n_adv + i;
@@ -415,7 +538,7 @@ int harvest(bsr_ctx *c, bsr_req *q, uint32_t r, uint32_t i) {
     else
       rc = (v == 2u) ? BSR_ERR_CHECKSUM : BSR_ERR_TRANSFER;
   }
-  if (rc == BSR_OK) c->st.bytes_installed[r] += c->chunk_bytes;
+  if (rc == BSR_OK) sd.bytes_installed[r] += c->chunk_bytes;
   return rc;
 }
 
@@ -430,8 +553,8 @@ int wait_event_deadline(bsr_ctx *c, cudaEvent_t ev, Clock::time_point deadline) 
 }
 
 // ---- restore when every advertised chunk already lives in device memory --------------------------
-int restore_resident(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_point deadline,
-                     const std::vector<TierObj> &objs) {
+int restore_resident(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
+                     Clock::time_point deadline, const std::vector<TierObj> &objs, StatDelta &sd) {
   const uint32_t R = c->cfg.n_ranks, W = c->cfg.window_chunks, N = q->n_adv;
   const uint32_t per_launch = BSR_K_MAX_BATCH / R ? BSR_K_MAX_BATCH / R : 1;
   int rc = BSR_OK;
@@ -448,112 +571,117 @@ int restore_resident(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_po
     }
   CU(c, cudaMemcpyAsync(q->d_desc, q->h_desc, (size_t)N * R * sizeof(BsrChunkDesc),
                         cudaMemcpyHostToDevice, stream));
-  c->st.h2d_copies++;
+  sd.h2d_copies++;
   // Nothing is staged for device-resident objects, so a window bounds nothing here: it is counted
   // (K = ceil(N / W)) and the launches take as many chunks as the kernel's scratch allows.
-  c->st.windows += (N + W - 1) / W;
-  {
-    const uint32_t w1 = N;
-    for (uint32_t b0 = 0; b0 < w1 && rc == BSR_OK; b0 += per_launch) {
-      const uint32_t b1 = (b0 + per_launch < w1) ? b0 + per_launch : w1;
-      BsrInstallParams p{};
-      fill_params(c, p, (uint32_t)(c->launch_seq++ % kLaunchSlots));
-      p.n_adv = N;
-      p.scatter = 1;
-      p.tables = q->d_table_ptrs;
-      p.ck_out = q->d_ck;
-      p.verdict = q->d_verdict;
-      p.batch = q->d_desc + (size_t)b0 * R;
-      p.n_chunks = (b1 - b0) * R;
-      if (c->cfg.time_kernels) {
-        if (n_timed == c->ev_pool.size()) {
-          cudaEvent_t e0 = nullptr, e1 = nullptr;
-          CU(c, cudaEventCreate(&e0));
-          CU(c, cudaEventCreate(&e1));
-          c->ev_pool.emplace_back(e0, e1);
-        }
-        CU(c, cudaEventRecord(c->ev_pool[n_timed].first, stream));
+  sd.windows += (N + W - 1) / W;
+  for (uint32_t b0 = 0; b0 < N && rc == BSR_OK; b0 += per_launch) {
+    const uint32_t b1 = (b0 + per_launch < N) ? b0 + per_launch : N;
+    BsrInstallParams p{};
+    fill_params(c, p, res, R * c->cfg.dev_staging_depth + (uint32_t)(res->seq++ % kLaunchSlots));
+    p.n_adv = N;
+    p.scatter = 1;
+    p.tables = q->d_table_ptrs;
+    p.ck_out = q->d_ck;
+    p.verdict = q->d_verdict;
+    p.batch = q->d_desc + (size_t)b0 * R;
+    p.n_chunks = (b1 - b0) * R;
+    if (c->cfg.time_kernels) {
+      if (n_timed == res->ev_pool.size()) {
+        cudaEvent_t e0 = nullptr, e1 = nullptr;
+        CU(c, cudaEventCreate(&e0));
+        CU(c, cudaEventCreate(&e1));
+        res->ev_pool.emplace_back(e0, e1);
       }
-      rc = launch_install(c, p, stream);
-      if (c->cfg.time_kernels) {
-        CU(c, cudaEventRecord(c->ev_pool[n_timed].second, stream));
-        ++n_timed;
-      }
+      CU(c, cudaEventRecord(res->ev_pool[n_timed].first, stream));
+    }
+    rc = launch_install(c, p, stream, sd);
+    if (c->cfg.time_kernels) {
+      CU(c, cudaEventRecord(res->ev_pool[n_timed].second, stream));
+      ++n_timed;
     }
   }
-  cudaEvent_t done = c->ev_done;
-  CU(c, cudaEventRecord(done, stream));
-  int wrc = wait_event_deadline(c, done, deadline);
-  if (wrc == BSR_ERR_TIMEOUT) {  // kernels are finite: let them finish, then report
-    cudaStreamSynchronize(stream);
-  }
+  CU(c, cudaEventRecord(res->ev_done, stream));
+  int wrc = wait_event_deadline(c, res->ev_done, deadline);
+  if (wrc == BSR_ERR_TIMEOUT) cudaStreamSynchronize(stream);  // kernels are finite: let them finish
   for (size_t k = 0; k < n_timed; ++k) {
     float ms = 0.f;
-    if (cudaEventElapsedTime(&ms, c->ev_pool[k].first, c->ev_pool[k].second) == cudaSuccess)
-      c->st.install_kernel_ms += ms;
+    if (cudaEventElapsedTime(&ms, res->ev_pool[k].first, res->ev_pool[k].second) == cudaSuccess)
+      sd.install_kernel_ms += ms;
   }
   if (rc == BSR_OK) rc = wrc;
   if (rc != BSR_OK) return rc;
   for (uint32_t i = 0; i < N; ++i)
     for (uint32_t r = 0; r < R; ++r) {
-      const int h = harvest(c, q, r, i);
+      const int h = harvest(c, q, r, i, sd);
       if (h != BSR_OK && rc == BSR_OK) rc = h;
     }
   return rc;
 }
 
-// ---- restore through the pinned ring --------------------------------------------------------------
-int restore_ring(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_point deadline) {
+// ---- restore through the pinned slot pool --------------------------------------------------------
+int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
+                 Clock::time_point deadline, StatDelta &sd) {
   int rc = ensure_ring(c);
   if (rc != BSR_OK) return rc;
   const uint32_t R = c->cfg.n_ranks, W = c->cfg.window_chunks, D = c->cfg.dev_staging_depth;
   const uint32_t N = q->n_adv, total = N * R;
   const uint32_t P = c->pieces;
   const bool direct = c->cfg.direct_install != 0;
-  std::vector<std::atomic<int>> state((size_t)total * P);  // per piece: 0 pending, 1 ready, <0 error
-  for (auto &s : state) s.store(0, std::memory_order_relaxed);
-  std::vector<TierObj> objs(total);
+  Job job;
+  job.q = q;
+  job.deadline = deadline;
+  job.P = P;
+  job.state.reset(new std::atomic<int>[(size_t)total * P]);
+  for (size_t k = 0; k < (size_t)total * P; ++k) job.state[k].store(0, std::memory_order_relaxed);
+  job.objs.resize(total);
+  job.slot.assign(total, 0);
   {
     std::lock_guard<std::mutex> lk(c->fill_mu);
-    c->cur_req = q;
-    c->fill_total = total * P;
-    c->fill_admitted = 0;
-    c->fill_next = 0;
-    c->fill_abort.store(false);
-    c->fill_deadline = deadline;
-    c->task_state = &state;
-    c->task_obj = &objs;
+    c->jobs.push_back(&job);
   }
   uint32_t admitted = 0, submitted = 0, reaped = 0, cur_piece = 0;
-  uint32_t released[BSR_MAX_RANKS] = {};
-  for (uint32_t r = 0; r < R; ++r) c->live[r] = 0;
+  uint32_t live[BSR_MAX_RANKS] = {};
   bool stop = false;  // a failure was seen: admit and submit nothing more, drain
 
   auto first_error = [&](int code) {
     if (rc == BSR_OK) rc = code;
     stop = true;
-    c->fill_abort.store(true, std::memory_order_release);
+    job.abort.store(true, std::memory_order_release);
+  };
+  auto release_slot = [&](uint32_t s) {
+    const uint32_t r = s % R;
+    std::lock_guard<std::mutex> pl(c->pool_mu);
+    c->free_slots[r].push_back(job.slot[s]);
+    c->live_total[r]--;
   };
 
   while (true) {
     bool progress = false;
-    // admit: chunk i of rank r enters the window as soon as slot i mod W is free (Eq. 3)
+    // admit: chunk i of rank r enters the window when this restore holds fewer than W slots of the
+    // rank (Eq. 3) and the pool, shared with the other restores in flight, has a free one
     if (!stop) {
       uint32_t n_new = 0;
       while (admitted < total) {
         const uint32_t i = admitted / R, r = admitted % R;
-        if (i - released[r] >= W) break;
-        if (i % W == 0 && r == 0) c->st.windows++;
-        c->live[r]++;
-        const uint64_t bytes = c->live[r] * c->slot_bytes;
-        if (bytes > c->st.peak_staging_bytes[r]) c->st.peak_staging_bytes[r] = bytes;
+        if (live[r] >= W) break;
+        {
+          std::lock_guard<std::mutex> pl(c->pool_mu);
+          if (c->free_slots[r].empty()) break;
+          job.slot[admitted] = c->free_slots[r].back();
+          c->free_slots[r].pop_back();
+          const uint64_t bytes = ++c->live_total[r] * c->slot_bytes;
+          if (bytes > c->st.peak_staging_bytes[r]) c->st.peak_staging_bytes[r] = bytes;
+        }
+        if (i % W == 0 && r == 0) sd.windows++;
+        live[r]++;
         ++admitted;
         ++n_new;
       }
       if (n_new) {
         {
           std::lock_guard<std::mutex> lk(c->fill_mu);
-          c->fill_admitted = admitted * P;
+          job.fill_admitted = admitted * P;
         }
         c->fill_cv.notify_all();
         progress = true;
@@ -562,22 +690,26 @@ int restore_ring(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_point 
     // reap, in order: observe the install of the oldest chunk in flight, release its slot
     while (reaped < submitted) {
       const uint32_t i = reaped / R, r = reaped % R, k = r * D + i % D;
-      cudaError_t e = cudaEventQuery(c->ev_inst[k]);
+      cudaError_t e = cudaEventQuery(res->ev_inst[k]);
       if (e == cudaErrorNotReady) break;
       if (e != cudaSuccess) {
         first_error(fail(c, BSR_ERR_CUDA, "install event: %s", cudaGetErrorString(e)));
-        reaped = submitted;  // the context is unusable; nothing more can be observed
+        while (reaped < submitted) {  // the context is unusable; nothing more can be observed
+          release_slot(reaped);
+          live[reaped % R]--;
+          ++reaped;
+        }
         break;
       }
       if (c->cfg.time_kernels) {
         float ms = 0.f;
-        if (cudaEventElapsedTime(&ms, c->ev_start[k], c->ev_inst[k]) == cudaSuccess)
-          c->st.install_kernel_ms += ms;
+        if (cudaEventElapsedTime(&ms, res->ev_start[k], res->ev_inst[k]) == cudaSuccess)
+          sd.install_kernel_ms += ms;
       }
-      const int h = harvest(c, q, r, i);
+      const int h = harvest(c, q, r, i, sd);
       if (h != BSR_OK) first_error(h);
-      c->live[r]--;
-      released[r] = i + 1;
+      release_slot(reaped);
+      live[r]--;
       ++reaped;
       progress = true;
     }
@@ -585,11 +717,12 @@ int restore_ring(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_point 
     // is complete, the install kernel on the compute stream
     while (!stop && submitted < admitted && submitted - reaped < R * D) {
       const uint32_t i = submitted / R, r = submitted % R, d = i % D, k = r * D + d;
-      uint8_t *stage = direct ? nullptr : c->dstage[r] + (size_t)d * c->chunk_bytes;
+      uint8_t *stage = direct ? nullptr : res->dstage[r] + (size_t)d * c->chunk_bytes;
+      uint8_t *slot_host = c->ring[r] + (size_t)job.slot[submitted] * c->slot_bytes;
       cudaError_t e = cudaSuccess;
       bool blocked = false;
       while (cur_piece < P) {
-        const int stt = state[(size_t)submitted * P + cur_piece].load(std::memory_order_acquire);
+        const int stt = job.state[(size_t)submitted * P + cur_piece].load(std::memory_order_acquire);
         if (stt == 0) {
           blocked = true;
           break;
@@ -598,40 +731,38 @@ int restore_ring(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_point 
           first_error(stt);
           break;
         }
-        const TierObj &o = objs[submitted];
+        const TierObj &o = job.objs[submitted];
         const uint64_t off = (uint64_t)cur_piece * kPieceBytes;
         const uint64_t len = (c->chunk_bytes - off < kPieceBytes) ? c->chunk_bytes - off : kPieceBytes;
-        const uint8_t *from = (o.loc == BSR_LOC_HOST)
-                                  ? c->ring[r] + (size_t)(i % W) * c->slot_bytes + off
-                                  : o.data + off;
+        const uint8_t *from = (o.loc == BSR_LOC_HOST) ? slot_host + off : o.data + off;
         if (!direct) {
-          if (cur_piece == 0) e = cudaStreamWaitEvent(c->copy_stream, c->ev_inst[k], 0);
+          if (cur_piece == 0) e = cudaStreamWaitEvent(c->copy_stream, res->ev_inst[k], 0);
           if (e == cudaSuccess)
             e = cudaMemcpyAsync(stage + off, from, len, cudaMemcpyDefault, c->copy_stream);
           if (e != cudaSuccess) {
             first_error(fail(c, BSR_ERR_TRANSFER, "copy submit: %s", cudaGetErrorString(e)));
             break;
           }
-          c->st.h2d_copies++;
+          sd.h2d_copies++;
         }
-        c->st.bytes_filled[r] += (o.loc == BSR_LOC_HOST) ? len : 0;
-        c->st.bytes_h2d[r] += len;  // bytes that cross the host link, by copy or by kernel loads
+        sd.bytes_filled[r] += (o.loc == BSR_LOC_HOST) ? len : 0;
+        sd.bytes_h2d[r] += len;  // bytes that cross the host link, by copy or by kernel loads
         ++cur_piece;
         progress = true;
       }
       if (stop || blocked) break;
-      const TierObj &o = objs[submitted];
+      const TierObj &o = job.objs[submitted];
       if (!direct) {
-        e = cudaEventRecord(c->ev_h2d[k], c->copy_stream);
-        if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, c->ev_h2d[k], 0);
+        e = cudaEventRecord(res->ev_h2d[k], c->copy_stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, res->ev_h2d[k], 0);
       }
-      if (e == cudaSuccess && c->cfg.time_kernels) e = cudaEventRecord(c->ev_start[k], stream);
+      if (e == cudaSuccess && c->cfg.time_kernels) e = cudaEventRecord(res->ev_start[k], stream);
       if (e != cudaSuccess) {
         first_error(fail(c, BSR_ERR_TRANSFER, "copy submit: %s", cudaGetErrorString(e)));
         break;
       }
       BsrInstallParams p{};
-      fill_params(c, p, (uint32_t)(c->launch_seq++ % kLaunchSlots));
+      fill_params(c, p, res, k);
       p.n_adv = N;
       p.scatter = 1;
       p.tables = q->d_table_ptrs;
@@ -640,13 +771,14 @@ int restore_ring(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_point 
       p.n_chunks = 1;
       // direct mode: the kernel reads the pinned slot (or the device object) itself over the link
       p.one.src = !direct ? stage
-                          : (o.loc == BSR_LOC_HOST ? c->ring_dev[r] + (size_t)(i % W) * c->slot_bytes
-                                                   : o.data);
+                          : (o.loc == BSR_LOC_HOST
+                                 ? c->ring_dev[r] + (size_t)job.slot[submitted] * c->slot_bytes
+                                 : o.data);
       p.one.chunk = i;
       p.one.rank = r;
       for (uint32_t g = 0; g < c->G; ++g) p.one.expect[g] = o.ck[g];
-      const int lrc = launch_install(c, p, stream, direct && o.loc == BSR_LOC_HOST);
-      e = cudaEventRecord(c->ev_inst[k], stream);
+      const int lrc = launch_install(c, p, stream, sd, direct && o.loc == BSR_LOC_HOST);
+      e = cudaEventRecord(res->ev_inst[k], stream);
       if (lrc != BSR_OK || e != cudaSuccess) {
         first_error(lrc != BSR_OK ? lrc : fail(c, BSR_ERR_CUDA, "record: %s", cudaGetErrorString(e)));
         break;
@@ -670,17 +802,112 @@ int restore_ring(bsr_ctx *c, bsr_req *q, cudaStream_t stream, Clock::time_point 
   // copies of a chunk that never reached its install launch may still be queued
   if (cur_piece != 0) cudaStreamSynchronize(c->copy_stream);
   // quiesce the fillers: nothing of this request may be touched after return
-  c->fill_abort.store(true, std::memory_order_release);
+  job.abort.store(true, std::memory_order_release);
   {
     std::unique_lock<std::mutex> lk(c->fill_mu);
-    c->fill_admitted = c->fill_next;  // hand out no further task
-    c->fill_cv.wait(lk, [&] { return c->fill_active == 0; });
-    c->cur_req = nullptr;
-    c->task_state = nullptr;
-    c->task_obj = nullptr;
+    job.fill_admitted = job.fill_next;  // hand out no further task
+    c->fill_cv.wait(lk, [&] { return job.fill_active == 0; });
+    for (size_t k = 0; k < c->jobs.size(); ++k)
+      if (c->jobs[k] == &job) {
+        c->jobs.erase(c->jobs.begin() + k);
+        break;
+      }
+    c->rr = 0;
   }
-  for (uint32_t r = 0; r < R; ++r) c->live[r] = 0;
+  // slots admitted but never installed go back to the pool
+  for (uint32_t s = reaped; s < admitted; ++s) release_slot(s);
   return rc;
+}
+
+// Shared by bsr_probe (tier 0, no request identity) and bsr_probe_request (all available tiers,
+// force-local marker).  request_scoped selects the second behaviour.
+int probe_impl(bsr_ctx *c, bool request_scoped, uint64_t request_id, const int32_t *tok,
+               size_t n_tok, int tok_on_device, uint64_t salt, uint64_t *keys_out,
+               uint64_t *hit_bitmap_out, uint32_t *n_hit_chunks, int *tier_out) {
+  if (!c || (!tok && n_tok) || !n_hit_chunks) return BSR_ERR_INVALID;
+  if (tier_out) *tier_out = -1;
+  const size_t N = n_tok / BSR_CHUNK_TOKENS;
+  if (N > (1u << 24)) return fail(c, BSR_ERR_INVALID, "probe: more than 2^24 chunks");
+  if (tok_on_device && (reinterpret_cast<uintptr_t>(tok) & 15u))
+    return fail(c, BSR_ERR_ALIGN, "probe: device token ids must be 16-byte aligned");
+  if (N == 0) {
+    *n_hit_chunks = 0;
+    return BSR_OK;
+  }
+  std::lock_guard<std::mutex> al(c->aux_mu);  // probe scratch is per context
+  CU(c, cudaSetDevice(c->cfg.device));
+  if (N > c->probe_cap_chunks) {
+    cudaFree(c->d_tok);
+    cudaFree(c->d_digests);
+    cudaFree(c->d_keys);
+    if (c->h_keys) cudaFreeHost(c->h_keys);
+    c->d_tok = nullptr;
+    c->d_digests = c->d_keys = c->h_keys = nullptr;
+    c->probe_cap_chunks = 0;
+    const size_t cap = round_up(N, 1024);
+    CU(c, cudaMalloc((void **)&c->d_tok, cap * BSR_CHUNK_TOKENS * 4));
+    CU(c, cudaMalloc((void **)&c->d_digests, cap * 8));
+    CU(c, cudaMalloc((void **)&c->d_keys, cap * 8));
+    CU(c, cudaHostAlloc((void **)&c->h_keys, cap * 8, cudaHostAllocDefault));
+    c->probe_cap_chunks = cap;
+  }
+  const int32_t *d_tok = tok;
+  cudaStream_t s = c->own_stream;
+  if (!tok_on_device) {
+    CU(c, cudaMemcpyAsync(c->d_tok, tok, N * BSR_CHUNK_TOKENS * 4, cudaMemcpyHostToDevice, s));
+    d_tok = c->d_tok;
+  }
+  // k_-1 = mix64(salt ^ mix64(reg_id)); a scalar, computed once per call
+  auto mix = [](uint64_t x) {
+    x += BSR_K_PHI;
+    x = (x ^ (x >> 32)) * BSR_K_PHI;
+    x = (x ^ (x >> 29)) * BSR_K_PHI;
+    return x ^ (x >> 32);
+  };
+  const uint64_t k_init = mix(salt ^ mix(c->cfg.reg_id));
+  const uint32_t per_block = BSR_K_PROBE_THREADS / 32;
+  const uint32_t grid = (uint32_t)((N + per_block - 1) / per_block);
+  bsr_probe_kernel<<<grid, BSR_K_PROBE_THREADS, 0, s>>>(d_tok, (uint32_t)N, salt, k_init,
+                                                        c->d_digests, c->d_probe_cnt, c->d_keys);
+  CU(c, cudaGetLastError());
+  CU(c, cudaMemcpyAsync(c->h_keys, c->d_keys, N * 8, cudaMemcpyDeviceToHost, s));
+  CU(c, cudaStreamSynchronize(s));
+  // index lookup: keys only; no payload byte is read, nothing is pinned or referenced afterwards
+  const size_t words = (N + 63) / 64;
+  if (hit_bitmap_out) memset(hit_bitmap_out, 0, words * 8);
+  uint32_t best_n = 0;
+  int best_tier = -1;
+  {
+    std::lock_guard<std::mutex> lk(c->mu);
+    c->st.kernel_launches++;
+    const bool forced = request_scoped && c->force_local.count(request_id) != 0;
+    std::vector<uint64_t> bm(words), best_bm(words, 0ull);
+    for (uint32_t t = 0; t < BSR_MAX_TIERS && !forced; ++t) {
+      if (request_scoped ? !c->tier_available[t] : t != 0) continue;
+      std::fill(bm.begin(), bm.end(), 0ull);
+      uint32_t n_hit = 0;
+      bool prefix = true;
+      for (size_t i = 0; i < N; ++i) {
+        bool hit = true;
+        for (uint32_t r = 0; r < c->cfg.n_ranks && hit; ++r)
+          hit = c->tier[t][r].find(c->h_keys[i]) != c->tier[t][r].end();
+        if (hit) bm[i / 64] |= 1ull << (i % 64);
+        if (!hit) prefix = false;
+        if (prefix) ++n_hit;
+      }
+      // one tier serves the request: the longest complete prefix, the higher-priority tier on a tie
+      if (n_hit > best_n || (!request_scoped && t == 0)) {
+        best_n = n_hit;
+        best_tier = n_hit ? (int)t : -1;
+        best_bm = bm;
+      }
+    }
+    if (hit_bitmap_out) memcpy(hit_bitmap_out, best_bm.data(), words * 8);
+  }
+  if (keys_out) memcpy(keys_out, c->h_keys, N * 8);
+  *n_hit_chunks = best_n;
+  if (tier_out) *tier_out = best_tier;
+  return BSR_OK;
 }
 
 }  // namespace
@@ -712,23 +939,19 @@ int bsr_ctx_create(const bsr_config *cfg, bsr_ctx **out) {
   if (c->cfg.dev_staging_depth > 16) c->cfg.dev_staging_depth = 16;
   if (c->cfg.timeout_ms == 0) c->cfg.timeout_ms = 30000;
   if (c->cfg.slot_align == 0) c->cfg.slot_align = 4096;
-  const size_t acc_bytes = (size_t)kLaunchSlots * BSR_K_MAX_BATCH * BSR_K_MAX_GROUPS * 8;
-  const size_t cnt_bytes = (kLaunchSlots + 2) * sizeof(unsigned int);
+  c->budget = c->cfg.budget_slots ? c->cfg.budget_slots : c->cfg.window_chunks;
   bool ok = cudaSetDevice(cfg->device) == cudaSuccess &&
             cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess &&
             cudaStreamCreateWithFlags(&c->own_stream, cudaStreamNonBlocking) == cudaSuccess &&
-            cudaEventCreateWithFlags(&c->ev_done, cudaEventDisableTiming) == cudaSuccess &&
-            cudaMalloc(&c->d_acc, acc_bytes) == cudaSuccess &&
-            cudaMalloc(&c->d_counters, cnt_bytes) == cudaSuccess &&
-            cudaMemset(c->d_acc, 0, acc_bytes) == cudaSuccess &&
-            cudaMemset(c->d_counters, 0, cnt_bytes) == cudaSuccess &&
+            init_scratch(c, &c->aux, kLaunchSlots) == BSR_OK &&
+            cudaMalloc(&c->d_probe_cnt, sizeof(unsigned int)) == cudaSuccess &&
+            cudaMemset(c->d_probe_cnt, 0, sizeof(unsigned int)) == cudaSuccess &&
             cudaDeviceSynchronize() == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
     bsr_ctx_destroy(c);
     return BSR_ERR_CUDA;
   }
-  c->st.dev_aux_bytes = acc_bytes + cnt_bytes;
   *out = c;
   return BSR_OK;
 }
@@ -743,18 +966,13 @@ int bsr_ctx_destroy(bsr_ctx *c) {
   c->fill_cv.notify_all();
   for (auto &t : c->fillers) t.join();
   cudaDeviceSynchronize();
-  for (uint32_t r = 0; r < BSR_MAX_RANKS; ++r) {
+  for (uint32_t r = 0; r < BSR_MAX_RANKS; ++r)
     if (c->ring[r]) cudaFreeHost(c->ring[r]);
-    if (c->dstage[r]) cudaFree(c->dstage[r]);
+  for (JobRes *res : c->res_all) {
+    destroy_res(res);
+    delete res;
   }
-  for (auto e : c->ev_h2d) cudaEventDestroy(e);
-  for (auto e : c->ev_inst) cudaEventDestroy(e);
-  for (auto e : c->ev_start) cudaEventDestroy(e);
-  for (auto &pr : c->ev_pool) {
-    cudaEventDestroy(pr.first);
-    cudaEventDestroy(pr.second);
-  }
-  if (c->ev_done) cudaEventDestroy(c->ev_done);
+  destroy_res(&c->aux);
   cudaFree(c->d_tiles);
   cudaFree(c->d_tensor_base);
   cudaFree(c->d_tensor_group);
@@ -762,8 +980,7 @@ int bsr_ctx_destroy(bsr_ctx *c) {
   cudaFree(c->d_put_stage);
   if (c->h_put_ck) cudaFreeHost(c->h_put_ck);
   if (c->h_put_verdict) cudaFreeHost(c->h_put_verdict);
-  cudaFree(c->d_acc);
-  cudaFree(c->d_counters);
+  cudaFree(c->d_probe_cnt);
   cudaFree(c->d_tok);
   cudaFree(c->d_digests);
   cudaFree(c->d_keys);
@@ -783,7 +1000,7 @@ int bsr_register(bsr_ctx *c, uint32_t rank, const bsr_group_desc *groups, uint32
   if (rank >= c->cfg.n_ranks || n_groups == 0 || n_groups > BSR_MAX_GROUPS || n_tensors == 0 ||
       n_tensors > 65535)
     return fail(c, BSR_ERR_INVALID, "register: rank/groups/tensors out of range");
-  if (c->finalized) return fail(c, BSR_ERR_STATE, "register after the registration was used");
+  if (c->finalized.load()) return fail(c, BSR_ERR_STATE, "register after the registration was used");
   for (uint32_t g = 0; g < n_groups; ++g) {
     const uint32_t B = groups[g].block_tokens;
     if (B == 0 || BSR_CHUNK_TOKENS % B || BSR_CHUNK_TOKENS / B > 255 || groups[g].num_phys_blocks == 0)
@@ -880,10 +1097,10 @@ int bsr_tier_put_at(bsr_ctx *c, uint32_t tier, uint32_t rank, uint64_t key, cons
     for (uint32_t g = 0; g < c->G; ++g) o.ck[g] = group_ck[g];
   } else {
     // store path: compute the group checksums on the GPU with the install kernel's sum stage
-    std::lock_guard<std::mutex> rl(c->restore_mu);
     CU(c, cudaSetDevice(c->cfg.device));
-    int rc = finalize_registration(c);
+    int rc = ensure_finalized(c);
     if (rc != BSR_OK) return rc;
+    std::lock_guard<std::mutex> al(c->aux_mu);
     if (!c->h_put_ck) {
       CU(c, cudaHostAlloc((void **)&c->h_put_ck, BSR_MAX_GROUPS * 8, cudaHostAllocMapped));
       CU(c, cudaHostAlloc((void **)&c->h_put_verdict, BSR_MAX_GROUPS * 4, cudaHostAllocMapped));
@@ -897,16 +1114,18 @@ int bsr_tier_put_at(bsr_ctx *c, uint32_t tier, uint32_t rank, uint64_t key, cons
       src = c->d_put_stage;
     }
     BsrInstallParams p{};
-    fill_params(c, p, (uint32_t)(c->launch_seq++ % kLaunchSlots));
+    fill_params(c, p, &c->aux, (uint32_t)(c->aux.seq++ % kLaunchSlots));
     p.n_adv = 1;
     p.scatter = 0;
     p.ck_out = c->d_put_ck;
     p.verdict = c->d_put_verdict;
     p.n_chunks = 1;
     p.one.src = src;
-    rc = launch_install(c, p, c->own_stream);
+    StatDelta sd;
+    rc = launch_install(c, p, c->own_stream, sd);
     if (rc != BSR_OK) return rc;
     CU(c, cudaStreamSynchronize(c->own_stream));
+    merge_stats(c, sd);
     for (uint32_t g = 0; g < c->G; ++g) o.ck[g] = c->h_put_ck[g];
   }
   std::lock_guard<std::mutex> lk(c->mu);
@@ -941,98 +1160,6 @@ int bsr_tier_checksums(bsr_ctx *c, uint32_t rank, uint64_t key, uint64_t *out) {
   return BSR_OK;
 }
 
-// Shared by bsr_probe (tier 0, no request identity) and bsr_probe_request (all available tiers,
-// force-local marker).  request_scoped selects the second behaviour.
-static int probe_impl(bsr_ctx *c, bool request_scoped, uint64_t request_id, const int32_t *tok,
-                      size_t n_tok, int tok_on_device, uint64_t salt, uint64_t *keys_out,
-                      uint64_t *hit_bitmap_out, uint32_t *n_hit_chunks, int *tier_out) {
-  if (!c || (!tok && n_tok) || !n_hit_chunks) return BSR_ERR_INVALID;
-  if (tier_out) *tier_out = -1;
-  const size_t N = n_tok / BSR_CHUNK_TOKENS;
-  if (N > (1u << 24)) return fail(c, BSR_ERR_INVALID, "probe: more than 2^24 chunks");
-  if (tok_on_device && (reinterpret_cast<uintptr_t>(tok) & 15u))
-    return fail(c, BSR_ERR_ALIGN, "probe: device token ids must be 16-byte aligned");
-  if (N == 0) {
-    *n_hit_chunks = 0;
-    return BSR_OK;
-  }
-  std::lock_guard<std::mutex> rl(c->restore_mu);  // probe scratch is per context
-  CU(c, cudaSetDevice(c->cfg.device));
-  if (N > c->probe_cap_chunks) {
-    cudaFree(c->d_tok);
-    cudaFree(c->d_digests);
-    cudaFree(c->d_keys);
-    if (c->h_keys) cudaFreeHost(c->h_keys);
-    c->d_tok = nullptr;
-    c->d_digests = c->d_keys = c->h_keys = nullptr;
-    c->probe_cap_chunks = 0;
-    const size_t cap = round_up(N, 1024);
-    CU(c, cudaMalloc((void **)&c->d_tok, cap * BSR_CHUNK_TOKENS * 4));
-    CU(c, cudaMalloc((void **)&c->d_digests, cap * 8));
-    CU(c, cudaMalloc((void **)&c->d_keys, cap * 8));
-    CU(c, cudaHostAlloc((void **)&c->h_keys, cap * 8, cudaHostAllocDefault));
-    c->probe_cap_chunks = cap;
-  }
-  const int32_t *d_tok = tok;
-  cudaStream_t s = c->own_stream;
-  if (!tok_on_device) {
-    CU(c, cudaMemcpyAsync(c->d_tok, tok, N * BSR_CHUNK_TOKENS * 4, cudaMemcpyHostToDevice, s));
-    d_tok = c->d_tok;
-  }
-  // k_-1 = mix64(salt ^ mix64(reg_id)); a scalar, computed once per call
-  auto mix = [](uint64_t x) {
-    x += BSR_K_PHI;
-    x = (x ^ (x >> 32)) * BSR_K_PHI;
-    x = (x ^ (x >> 29)) * BSR_K_PHI;
-    return x ^ (x >> 32);
-  };
-  const uint64_t k_init = mix(salt ^ mix(c->cfg.reg_id));
-  const uint32_t per_block = BSR_K_PROBE_THREADS / 32;
-  const uint32_t grid = (uint32_t)((N + per_block - 1) / per_block);
-  bsr_probe_kernel<<<grid, BSR_K_PROBE_THREADS, 0, s>>>(d_tok, (uint32_t)N, salt, k_init,
-                                                        c->d_digests, c->d_counters + kLaunchSlots,
-                                                        c->d_keys);
-  CU(c, cudaGetLastError());
-  c->st.kernel_launches++;
-  CU(c, cudaMemcpyAsync(c->h_keys, c->d_keys, N * 8, cudaMemcpyDeviceToHost, s));
-  CU(c, cudaStreamSynchronize(s));
-  // index lookup: keys only; no payload byte is read, nothing is pinned or referenced afterwards
-  const size_t words = (N + 63) / 64;
-  if (hit_bitmap_out) memset(hit_bitmap_out, 0, words * 8);
-  uint32_t best_n = 0;
-  int best_tier = -1;
-  {
-    std::lock_guard<std::mutex> lk(c->mu);
-    const bool forced = request_scoped && c->force_local.count(request_id) != 0;
-    std::vector<uint64_t> bm(words), best_bm(words, 0ull);
-    for (uint32_t t = 0; t < BSR_MAX_TIERS && !forced; ++t) {
-      if (request_scoped ? !c->tier_available[t] : t != 0) continue;
-      std::fill(bm.begin(), bm.end(), 0ull);
-      uint32_t n_hit = 0;
-      bool prefix = true;
-      for (size_t i = 0; i < N; ++i) {
-        bool hit = true;
-        for (uint32_t r = 0; r < c->cfg.n_ranks && hit; ++r)
-          hit = c->tier[t][r].find(c->h_keys[i]) != c->tier[t][r].end();
-        if (hit) bm[i / 64] |= 1ull << (i % 64);
-        if (!hit) prefix = false;
-        if (prefix) ++n_hit;
-      }
-      // one tier serves the request: the longest complete prefix, the higher-priority tier on a tie
-      if (n_hit > best_n || (!request_scoped && t == 0)) {
-        best_n = n_hit;
-        best_tier = n_hit ? (int)t : -1;
-        best_bm = bm;
-      }
-    }
-    if (hit_bitmap_out) memcpy(hit_bitmap_out, best_bm.data(), words * 8);
-  }
-  if (keys_out) memcpy(keys_out, c->h_keys, N * 8);
-  *n_hit_chunks = best_n;
-  if (tier_out) *tier_out = best_tier;
-  return BSR_OK;
-}
-
 int bsr_probe(bsr_ctx *c, const int32_t *tok, size_t n_tok, int tok_on_device, uint64_t salt,
               uint64_t *keys_out, uint64_t *hit_bitmap_out, uint32_t *n_hit_chunks) {
   return probe_impl(c, false, 0, tok, n_tok, tok_on_device, salt, keys_out, hit_bitmap_out,
@@ -1048,7 +1175,7 @@ int bsr_probe_request(bsr_ctx *c, uint64_t request_id, const int32_t *tok, size_
 
 int bsr_req_bind(bsr_ctx *c, bsr_req *q, uint64_t request_id, uint32_t tier) {
   if (!c || !q || q->ctx != c || tier >= BSR_MAX_TIERS) return BSR_ERR_INVALID;
-  std::lock_guard<std::mutex> rl(c->restore_mu);
+  std::lock_guard<std::mutex> ql(q->mu);
   q->request_id = request_id;
   q->tier = tier;
   q->bound = true;
@@ -1072,10 +1199,9 @@ int bsr_request_is_force_local(bsr_ctx *c, uint64_t request_id, int *out) {
 int bsr_req_create(bsr_ctx *c, const uint64_t *keys, uint32_t n_adv, const int32_t *const *tables,
                    bsr_req **out) {
   if (!c || !out || (n_adv && (!keys || !tables))) return BSR_ERR_INVALID;
+  CU(c, cudaSetDevice(c->cfg.device));
   {
-    std::lock_guard<std::mutex> rl(c->restore_mu);
-    CU(c, cudaSetDevice(c->cfg.device));
-    int rc = finalize_registration(c);
+    int rc = ensure_finalized(c);
     if (rc != BSR_OK) return rc;
   }
   const uint32_t R = c->cfg.n_ranks, G = c->G;
@@ -1113,7 +1239,6 @@ int bsr_req_create(bsr_ctx *c, const uint64_t *keys, uint32_t n_adv, const int32
     bsr_req_release(c, q);
     return fail(c, code, "req_create: %s", what);
   };
-  cudaSetDevice(c->cfg.device);
   if (n_adv) {
     if (cudaMalloc((void **)&q->d_tables, total_entries * 4) != cudaSuccess ||
         cudaMalloc((void **)&q->d_table_ptrs, (size_t)R * G * sizeof(void *)) != cudaSuccess)
@@ -1140,7 +1265,8 @@ int bsr_req_create(bsr_ctx *c, const uint64_t *keys, uint32_t n_adv, const int32
     memset(q->h_ck, 0, cells * 8);
     memset(q->h_verdict, 0, cells * 4);
     const size_t n_desc = (size_t)R * n_adv;
-    if (cudaHostAlloc((void **)&q->h_desc, n_desc * sizeof(BsrChunkDesc), cudaHostAllocDefault) != cudaSuccess ||
+    if (cudaHostAlloc((void **)&q->h_desc, n_desc * sizeof(BsrChunkDesc), cudaHostAllocDefault) !=
+            cudaSuccess ||
         cudaMalloc((void **)&q->d_desc, n_desc * sizeof(BsrChunkDesc)) != cudaSuccess)
       return bail(BSR_ERR_NOMEM, "descriptor arrays");
   }
@@ -1150,7 +1276,7 @@ int bsr_req_create(bsr_ctx *c, const uint64_t *keys, uint32_t n_adv, const int32
 
 int bsr_req_release(bsr_ctx *c, bsr_req *q) {
   if (!c || !q || q->ctx != c) return BSR_ERR_INVALID;
-  std::lock_guard<std::mutex> rl(c->restore_mu);
+  { std::lock_guard<std::mutex> ql(q->mu); }  // wait for a call in flight on this request
   cudaSetDevice(c->cfg.device);
   cudaFree(q->d_tables);
   cudaFree(q->d_table_ptrs);
@@ -1165,21 +1291,23 @@ int bsr_req_release(bsr_ctx *c, bsr_req *q) {
 
 int bsr_restore(bsr_ctx *c, bsr_req *q, void *cuda_stream) {
   if (!c || !q || q->ctx != c) return BSR_ERR_INVALID;
-  std::lock_guard<std::mutex> rl(c->restore_mu);  // bounded-retrieve lock
+  std::lock_guard<std::mutex> ql(q->mu);
+  // the bounded-retrieve lock; with an admission budget restores share the slot pool instead
+  std::unique_lock<std::mutex> serial(c->restore_mu, std::defer_lock);
+  if (c->cfg.budget_slots == 0) serial.lock();
   const auto t0 = Clock::now();
   const auto deadline = t0 + std::chrono::milliseconds(c->cfg.timeout_ms);
   CU(c, cudaSetDevice(c->cfg.device));
-  cudaStream_t stream = cuda_stream ? static_cast<cudaStream_t>(cuda_stream) : c->own_stream;
-  clear_request_state(q);
+  std::fill(q->bitmap.begin(), q->bitmap.end(), 0ull);
+  q->restored = false;
   q->failed = false;
   const uint32_t R = c->cfg.n_ranks, N = q->n_adv;
-  uint64_t installed_before[BSR_MAX_RANKS];
-  for (uint32_t r = 0; r < BSR_MAX_RANKS; ++r) installed_before[r] = c->st.bytes_installed[r];
   if (N) {
     const size_t cells = (size_t)R * c->G * N;
     memset(q->h_ck, 0, cells * 8);
     memset(q->h_verdict, 0, cells * 4);
   }
+  StatDelta sd;
   int rc = BSR_OK;
   bool tier_up;
   {
@@ -1189,55 +1317,63 @@ int bsr_restore(bsr_ctx *c, bsr_req *q, void *cuda_stream) {
   if (!tier_up) {
     rc = fail(c, BSR_ERR_TRANSFER, "tier %u is unavailable", q->tier);
   } else if (N) {
-    // are all advertised chunks already in device memory?  (then no staging is needed at all)
-    std::vector<TierObj> objs((size_t)N * R);
-    bool all_device = true;
-    {
-      std::lock_guard<std::mutex> lk(c->mu);
-      for (uint32_t i = 0; i < N && all_device; ++i)
-        for (uint32_t r = 0; r < R; ++r) {
-          auto it = c->tier[q->tier][r].find(q->keys[i]);
-          if (!c->tier_available[q->tier] || it == c->tier[q->tier][r].end() ||
-              it->second.loc != BSR_LOC_DEVICE) {
-            all_device = false;
-            break;
+    JobRes *res = nullptr;
+    rc = acquire_res(c, &res);
+    if (rc == BSR_OK) {
+      cudaStream_t stream = cuda_stream ? static_cast<cudaStream_t>(cuda_stream) : res->stream;
+      // are all advertised chunks already in device memory?  (then no staging is needed at all)
+      std::vector<TierObj> objs((size_t)N * R);
+      bool all_device = true;
+      {
+        std::lock_guard<std::mutex> lk(c->mu);
+        for (uint32_t i = 0; i < N && all_device; ++i)
+          for (uint32_t r = 0; r < R; ++r) {
+            auto it = c->tier[q->tier][r].find(q->keys[i]);
+            if (it == c->tier[q->tier][r].end() || it->second.loc != BSR_LOC_DEVICE) {
+              all_device = false;
+              break;
+            }
+            objs[(size_t)i * R + r] = it->second;
           }
-          objs[(size_t)i * R + r] = it->second;
+      }
+      rc = all_device ? restore_resident(c, q, res, stream, deadline, objs, sd)
+                      : restore_ring(c, q, res, stream, deadline, sd);
+      if (c->cfg.install_variant != BSR_INSTALL_VECTOR) {
+        // a bounded wait inside the bulk kernel that gave up raised the device-side error flag
+        unsigned int flag = 0;
+        unsigned int *d_flag = res->d_cnt + res->n_slots;
+        if (cudaMemcpy(&flag, d_flag, sizeof flag, cudaMemcpyDeviceToHost) != cudaSuccess) {
+          if (rc == BSR_OK) rc = fail(c, BSR_ERR_CUDA, "reading the kernel error flag failed");
+        } else if (flag) {
+          cudaMemset(d_flag, 0, sizeof flag);
+          if (rc == BSR_OK || rc == BSR_ERR_CHECKSUM)
+            rc = fail(c, BSR_ERR_TIMEOUT, "a bounded wait inside the install kernel gave up");
         }
-    }
-    rc = all_device ? restore_resident(c, q, stream, deadline, objs)
-                    : restore_ring(c, q, stream, deadline);
-  }
-  if (N && c->cfg.install_variant != BSR_INSTALL_VECTOR) {
-    // a bounded wait inside the bulk kernel that gave up raised the device-side error flag
-    unsigned int flag = 0;
-    unsigned int *d_flag = c->d_counters + kLaunchSlots + 1;
-    if (cudaMemcpy(&flag, d_flag, sizeof flag, cudaMemcpyDeviceToHost) != cudaSuccess) {
-      if (rc == BSR_OK) rc = fail(c, BSR_ERR_CUDA, "reading the kernel error flag failed");
-    } else if (flag) {
-      cudaMemset(d_flag, 0, sizeof flag);
-      if (rc == BSR_OK || rc == BSR_ERR_CHECKSUM)
-        rc = fail(c, BSR_ERR_TIMEOUT, "a bounded wait inside the install kernel gave up");
+      }
+      release_res(c, res);
+    } else if (res) {
+      release_res(c, res);  // partly built: kept in the pool's list for destruction only
     }
   }
-  if (rc == BSR_OK) {
+  if (rc == BSR_OK)
     q->restored = true;
-  } else {
+  else
     invalidate_host(q);
-    if (q->bound) {  // the next admission pass of this request must not re-enter the same fault
-      std::lock_guard<std::mutex> lk(c->mu);
+  merge_stats(c, sd);
+  {
+    std::lock_guard<std::mutex> lk(c->mu);
+    if (rc != BSR_OK && q->bound)  // the next admission pass must not re-enter the same fault
       c->force_local.insert(q->request_id);
-    }
+    for (uint32_t r = 0; r < R; ++r) c->st.bytes_restored_by_tier[q->tier] += sd.bytes_installed[r];
+    c->inject.kind = BSR_INJECT_NONE;  // one shot
+    c->st.last_restore_ms = std::chrono::duration<double, std::milli>(Clock::now() - t0).count();
   }
-  for (uint32_t r = 0; r < R; ++r) c->st.bytes_restored_by_tier[q->tier] += c->st.bytes_installed[r] - installed_before[r];
-  c->inject.kind = BSR_INJECT_NONE;  // one shot
-  c->st.last_restore_ms = std::chrono::duration<double, std::milli>(Clock::now() - t0).count();
   return rc;
 }
 
 int bsr_commit(bsr_ctx *c, bsr_req *q, uint32_t *exposed) {
   if (!c || !q || q->ctx != c || !exposed) return BSR_ERR_INVALID;
-  std::lock_guard<std::mutex> rl(c->restore_mu);
+  std::lock_guard<std::mutex> ql(q->mu);
   bool all = q->restored && !q->failed;
   const uint32_t R = c->cfg.n_ranks;
   for (uint32_t rg = 0; all && rg < R * c->G; ++rg)
@@ -1257,9 +1393,10 @@ int bsr_commit(bsr_ctx *c, bsr_req *q, uint32_t *exposed) {
 
 int bsr_invalidate(bsr_ctx *c, bsr_req *q, unsigned flags) {
   if (!c || !q || q->ctx != c) return BSR_ERR_INVALID;
-  std::lock_guard<std::mutex> rl(c->restore_mu);
+  std::lock_guard<std::mutex> ql(q->mu);
   invalidate_host(q);
   if ((flags & BSR_SCRUB) && q->n_adv) {
+    std::lock_guard<std::mutex> al(c->aux_mu);
     CU(c, cudaSetDevice(c->cfg.device));
     BsrScrubParams p{};
     p.tensor_base = c->d_tensor_base;
@@ -1278,8 +1415,9 @@ int bsr_invalidate(bsr_ctx *c, bsr_req *q, unsigned flags) {
     dim3 grid(max_logical < 1024 ? max_logical : 1024, c->cfg.n_ranks * c->L);
     bsr_scrub_kernel<<<grid, 256, 0, c->own_stream>>>(p);
     CU(c, cudaGetLastError());
-    c->st.kernel_launches++;
     CU(c, cudaStreamSynchronize(c->own_stream));
+    std::lock_guard<std::mutex> lk(c->mu);
+    c->st.kernel_launches++;
   }
   return BSR_OK;
 }
@@ -1287,7 +1425,7 @@ int bsr_invalidate(bsr_ctx *c, bsr_req *q, unsigned flags) {
 int bsr_req_bitmap(bsr_ctx *c, bsr_req *q, uint64_t *out, size_t words) {
   if (!c || !q || q->ctx != c || (!out && words)) return BSR_ERR_INVALID;
   if (words < q->bitmap.size()) return fail(c, BSR_ERR_INVALID, "bitmap buffer too small");
-  std::lock_guard<std::mutex> rl(c->restore_mu);
+  std::lock_guard<std::mutex> ql(q->mu);
   if (!q->bitmap.empty()) memcpy(out, q->bitmap.data(), q->bitmap.size() * 8);
   return BSR_OK;
 }
@@ -1296,21 +1434,23 @@ int bsr_req_checksums(bsr_ctx *c, bsr_req *q, uint64_t *out, size_t count) {
   if (!c || !q || q->ctx != c || (!out && count)) return BSR_ERR_INVALID;
   const size_t cells = (size_t)c->cfg.n_ranks * c->G * q->n_adv;
   if (count < cells) return fail(c, BSR_ERR_INVALID, "checksum buffer too small");
-  std::lock_guard<std::mutex> rl(c->restore_mu);
+  std::lock_guard<std::mutex> ql(q->mu);
   if (cells) memcpy(out, q->h_ck, cells * 8);
   return BSR_OK;
 }
 
 int bsr_get_stats(bsr_ctx *c, bsr_stats *out) {
   if (!c || !out) return BSR_ERR_INVALID;
-  std::lock_guard<std::mutex> rl(c->restore_mu);
+  std::lock_guard<std::mutex> pl(c->pool_mu);  // peak_staging_bytes is written under pool_mu
+  std::lock_guard<std::mutex> lk(c->mu);
   *out = c->st;
   return BSR_OK;
 }
 
 int bsr_reset_stats(bsr_ctx *c) {
   if (!c) return BSR_ERR_INVALID;
-  std::lock_guard<std::mutex> rl(c->restore_mu);
+  std::lock_guard<std::mutex> pl(c->pool_mu);
+  std::lock_guard<std::mutex> lk(c->mu);
   bsr_stats keep = c->st;
   c->st = bsr_stats{};
   c->st.slot_bytes = keep.slot_bytes;
@@ -1323,7 +1463,7 @@ int bsr_reset_stats(bsr_ctx *c) {
 int bsr_test_inject(bsr_ctx *c, int kind, uint32_t rank, uint32_t group, uint32_t chunk,
                     uint64_t seed) {
   if (!c || kind < BSR_INJECT_NONE || kind > BSR_INJECT_FILL_STALL) return BSR_ERR_INVALID;
-  std::lock_guard<std::mutex> rl(c->restore_mu);
+  std::lock_guard<std::mutex> lk(c->mu);
   c->inject.kind = kind;
   c->inject.rank = rank;
   c->inject.group = group;

@@ -103,3 +103,58 @@ def test_tier_lost_between_probe_and_restore_fails_closed():
     status, st = O.restore_request(eng, RID, tier, reg, req, paged, W)
     assert status == O.ERR_TRANSFER and O.commit(reg, req, paged) == 0 and RID in eng.force_local
     assert max(st.peak_staging_bytes) == 0
+
+
+# ---------------------------------------------------------------- admission budget B
+def _two_requests(N0, N1, corrupt=None):
+    """Two requests with different token streams restoring into the same pools (disjoint blocks)."""
+    layout = synth.tiny_layout()
+    reg = O.Registration(list(layout.block_tokens), list(layout.tensors))
+    Rk = 2
+    tiers = [O.Tier() for _ in range(Rk)]
+    Ns = [N0, N1]
+    pools = [synth.pool_blocks(layout, g, N0 + N1) for g in range(reg.n_groups)]
+    big = [[synth.block_table(layout, r, g, N0 + N1, seed=5) for g in range(reg.n_groups)] for r in range(Rk)]
+    reqs, payloads = [], {}
+    for k, N in enumerate(Ns):
+        tok = synth.tokens(N * 256, seed=100 + k)
+        keys = O.prefix_keys(O.chunk_digests(tok, 3), 3, 1)
+        for r in range(Rk):
+            for i in range(N):
+                p = synth.chunk_payload(layout, r, 1000 * k + i, seed=5).copy()
+                ck = O.group_checksums(reg, p)
+                if corrupt == (k, r, i):
+                    p[7] ^= 2
+                payloads[(k, r, i)] = p
+                tiers[r].put(keys[i], p, ck)
+        first = 0 if k == 0 else N0
+        tabs = [[big[r][g][first * reg.blocks_per_chunk(g):(first + N) * reg.blocks_per_chunk(g)]
+                 for g in range(reg.n_groups)] for r in range(Rk)]
+        reqs.append(O.Request(keys, tabs, Rk, reg.n_groups))
+    paged = [O.new_paged(reg, pools, synth.CANARY) for _ in range(Rk)]
+    return layout, reg, tiers, reqs, paged, payloads, pools
+
+
+def test_budget_bounds_aggregate_staging_and_results_equal_serial_restores():
+    for (W, B, want_peak_slots) in [(4, 6, 6), (4, 8, 8), (4, 16, 8), (4, 3, 3), (4, 4, 4)]:
+        layout, reg, tiers, reqs, paged, payloads, pools = _two_requests(11, 9)
+        status, peak, rounds = O.restore_concurrent(reg, tiers, reqs, paged, W, B)
+        assert status == [O.OK, O.OK]
+        assert peak == [want_peak_slots * reg.slot_bytes] * 2          # min(B, sum of windows)
+        assert [O.commit(reg, q, paged) for q in reqs] == [11, 9]
+        # the same two requests restored one after the other give the same bytes
+        layout, reg, tiers2, reqs2, paged2, _, _ = _two_requests(11, 9)
+        for q in reqs2:
+            assert O.restore(reg, tiers2, q, paged2, W)[0] == O.OK
+        for r in range(2):
+            for l in range(len(layout.tensors)):
+                assert np.array_equal(paged[r][l], paged2[r][l])
+
+
+def test_budget_one_request_fails_alone():
+    layout, reg, tiers, reqs, paged, payloads, pools = _two_requests(8, 8, corrupt=(1, 0, 5))
+    status, peak, rounds = O.restore_concurrent(reg, tiers, reqs, paged, 4, 6)
+    assert status == [O.OK, O.ERR_CHECKSUM]
+    assert O.commit(reg, reqs[0], paged) == 8 and O.commit(reg, reqs[1], paged) == 0
+    assert reqs[0].valid.all() and not reqs[1].valid.any()
+    assert max(peak) <= 6 * reg.slot_bytes
