@@ -308,7 +308,13 @@ def run_gpu(args):
                                  max(3, min(args.warmup, 3)), N)
     peak_staging = [int(st_e2e.peak_staging_bytes[r]) for r in range(R)]
     slot = int(st_e2e.slot_bytes)
+    e2e_install_us = 1e3 * st_e2e.install_kernel_ms / max(1, int(st_e2e.install_launches))
     clocks = sampler.stop()
+    # probe alone (token ids in host memory: H2D, digest + chain kernel, D2H of the keys, index lookup)
+    t0 = time.perf_counter()
+    for _ in range(20):
+        B.bsr_probe(e2e.ctx, tok, len(tok), salt, False)
+    probe_us = (time.perf_counter() - t0) / 20 * 1e6
     e2e.close()
 
     if rank != 0:
@@ -327,7 +333,8 @@ def run_gpu(args):
     traffic = NCU_DRAM_BYTES_PER_PAYLOAD_BYTE * per_launch_payload
 
     # ---- CPU oracle on a bounded sample -----------------------------------------------------
-    sample = 16
+    del payload  # 4.2 GB of host memory the oracle leg regenerates for itself
+    sample = min(N, 128)  # the whole workload: about 10-20 s of single-thread numpy work
     dt, nbytes = oracle_sample_step(layout, R, sample, W, seed)
     cpu = {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
            "sample": f"first {sample} of {N} chunks x {R} rank slices, one pass ({dt:.1f} s)"}
@@ -345,10 +352,12 @@ def run_gpu(args):
                                f"{args.load_concurrency}, dev_staging_depth={args.depth}"},
         "per_rank_GBps": value / (world * R),
         "restore_seconds": ms_res / 1e3,
+        "probe_host_us": probe_us,
         "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e, "steps": e2e_steps,
                 "h2d_bytes_per_step": step_bytes + len(tok) * 4,
                 "d2h_bytes_per_step": N * 8 + R * layout.n_groups * N * 12,
                 "per_rank_GBps": e2e_value / (world * R), "restore_seconds": ms_e2e / 1e3,
+                "install_us_per_chunk_launch": e2e_install_us,
                 "h2d_link_GBps_measured": h2d_gbs, "frac_of_h2d_link": e2e_value / world / h2d_gbs},
         "peak_staging_bytes_per_rank": peak_staging, "staging_law_bytes": W * slot,
         "staging_residual_bytes": [p - W * slot for p in peak_staging],

@@ -248,12 +248,17 @@ enum {
   BSR_INJECT_CORRUPT_SLOT = 1, /* flip one word of (rank, group, chunk) in the pinned slot after
                                   the fill, before the device copy                             */
   BSR_INJECT_FILL_ERROR = 2,   /* the tier read of (rank, chunk) reports a transfer error      */
-  BSR_INJECT_FILL_STALL = 3    /* the tier read of (rank, chunk) does not finish before the
+  BSR_INJECT_FILL_STALL = 3,   /* the tier read of (rank, chunk) does not finish before the
                                   deadline                                                     */
+  BSR_INJECT_KERNEL_WAIT = 4   /* in the install launch of (rank, chunk) one tile is never loaded and
+                                  the kernel's waits are bounded at 50 ms: the waits run out, the
+                                  kernel raises its error flag, drains and returns; the restore
+                                  reports BSR_ERR_TIMEOUT and the context stays usable           */
 };
 
-/* Arms one fault for the next restore (one shot; BSR_INJECT_NONE disarms).  Acts on host memory
- * and host threads only; the GPU is never made to fault, trap or spin. */
+/* Arms one fault for the next restore (one shot; BSR_INJECT_NONE disarms).  Kinds 1-3 act on host
+ * memory and host threads only.  Kind 4 makes a bounded wait inside the kernel expire; nothing is
+ * ever made to fault, trap or spin without a limit. */
 int bsr_test_inject(bsr_ctx *ctx, int kind, uint32_t rank, uint32_t group, uint32_t chunk,
                     uint64_t seed);
 

@@ -20,6 +20,7 @@ BSR_LOC_HOST, BSR_LOC_DEVICE = 0, 1
 BSR_INSTALL_AUTO, BSR_INSTALL_VECTOR, BSR_INSTALL_BULK = 0, 1, 2
 BSR_SCRUB = 1
 BSR_INJECT_NONE, BSR_INJECT_CORRUPT_SLOT, BSR_INJECT_FILL_ERROR, BSR_INJECT_FILL_STALL = 0, 1, 2, 3
+BSR_INJECT_KERNEL_WAIT = 4
 BSR_MAX_GROUPS, BSR_MAX_RANKS, BSR_CHUNK_TOKENS = 8, 8, 256
 
 ERROR_NAMES = {0: "BSR_OK", -1: "BSR_ERR_INVALID", -2: "BSR_ERR_MISSING", -3: "BSR_ERR_CHECKSUM",

@@ -54,6 +54,9 @@ struct BsrInstallParams {
   unsigned int *err_flag;    // set to nonzero if a bounded wait gave up (bulk variant)
   uint64_t *ck_out;          // [(r*G + g) * n_adv + i] computed checksum
   uint32_t *verdict;         // same index: 1 verified, 2 mismatch
+  uint64_t wait_ns;          // bound of every wait inside the bulk kernel; 0 = BSR_K_WAIT_NS
+  uint32_t stall_tile;       // test hook: work item whose load is never issued; ~0u = none
+  uint32_t pad0;
   const BsrChunkDesc *batch; // device array of n_chunks descriptors, or NULL: use `one`
   BsrChunkDesc one;          // the descriptor of a single-chunk launch, carried in the parameters
 };
@@ -261,13 +264,13 @@ __device__ __forceinline__ bool bsr_mbar_try_wait(uint32_t bar, uint32_t parity)
 }
 // Bounded wait.  Returns false if the deadline passed (and raises the error flag).
 __device__ __forceinline__ bool bsr_mbar_wait(uint32_t bar, uint32_t parity, unsigned int *err_flag,
-                                              volatile int *abort_flag) {
+                                              volatile int *abort_flag, uint64_t wait_ns) {
   if (bsr_mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = bsr_globaltimer();
   for (;;) {
     if (bsr_mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (bsr_globaltimer() - t0 > BSR_K_WAIT_NS) {
+    if (bsr_globaltimer() - t0 > wait_ns) {
       *abort_flag = 1;
       atomicExch(err_flag, 1u);
       return false;
@@ -318,6 +321,7 @@ bsr_install_bulk_kernel(const __grid_constant__ BsrInstallParams p) {
   }
   __syncthreads();
 
+  const uint64_t wait_ns = p.wait_ns ? p.wait_ns : BSR_K_WAIT_NS;
   // every byte is read once and written once: mark both streams evict-first in L2
   const uint64_t pol = bsr_policy_evict_first();
   const uint32_t total = p.n_chunks * p.n_tiles;
@@ -362,8 +366,10 @@ bsr_install_bulk_kernel(const __grid_constant__ BsrInstallParams p) {
           const uint32_t n = base + j;
           const uint32_t s = n % BSR_K_BULK_STAGES, round = n / BSR_K_BULK_STAGES;
           if (round > 0 &&
-              !bsr_mbar_wait(bsr_smem_u32(&empty_bar[s]), (round - 1) & 1u, p.err_flag, &abort_flag)) {
+              !bsr_mbar_wait(bsr_smem_u32(&empty_bar[s]), (round - 1) & 1u, p.err_flag, &abort_flag, wait_ns)) {
             ok = 0;
+          } else if (blockIdx.x + n * gridDim.x == p.stall_tile) {
+            // test hook: this tile's load is never issued, so the waits on its stage run out
           } else {
             meta[s].dst = dst_j;
             meta[s].bytes = bytes_j;
@@ -387,7 +393,7 @@ bsr_install_bulk_kernel(const __grid_constant__ BsrInstallParams p) {
       uint32_t n = 0;
       for (; n < my_tiles; ++n) {
         const uint32_t s = n % BSR_K_BULK_STAGES, round = n / BSR_K_BULK_STAGES;
-        if (!bsr_mbar_wait(bsr_smem_u32(&full_bar[s]), round & 1u, p.err_flag, &abort_flag)) break;
+        if (!bsr_mbar_wait(bsr_smem_u32(&full_bar[s]), round & 1u, p.err_flag, &abort_flag, wait_ns)) break;
         if (p.scatter) {
           bsr_bulk_store(meta[s].dst, bsr_smem_u32(stage_mem + (size_t)s * BSR_K_TILE_MAX),
                          meta[s].bytes, pol);
@@ -413,7 +419,7 @@ bsr_install_bulk_kernel(const __grid_constant__ BsrInstallParams p) {
     int cur_c = -1, cur_g = -1;
     for (uint32_t n = 0; n < my_tiles; ++n) {
       const uint32_t s = n % BSR_K_BULK_STAGES, round = n / BSR_K_BULK_STAGES;
-      if (!bsr_mbar_wait(bsr_smem_u32(&full_bar[s]), round & 1u, p.err_flag, &abort_flag)) break;
+      if (!bsr_mbar_wait(bsr_smem_u32(&full_bar[s]), round & 1u, p.err_flag, &abort_flag, wait_ns)) break;
       const BsrStageMeta m = meta[s];
       if (m.c != cur_c || m.g != cur_g) {  // warp-uniform
         if (cur_c >= 0) {
@@ -449,7 +455,7 @@ bsr_install_bulk_kernel(const __grid_constant__ BsrInstallParams p) {
       if (last_round[s] < 0) continue;
       const uint64_t t0 = bsr_globaltimer();
       while (!bsr_mbar_try_wait(bsr_smem_u32(&full_bar[s]), (uint32_t)last_round[s] & 1u) &&
-             bsr_globaltimer() - t0 < BSR_K_WAIT_NS / 8) {
+             bsr_globaltimer() - t0 < wait_ns) {
       }
     }
   }

@@ -285,6 +285,7 @@ void fill_params(bsr_ctx *c, BsrInstallParams &p, JobRes *res, uint32_t slot) {
   p.acc = res->d_acc + (size_t)slot * BSR_K_MAX_BATCH * BSR_K_MAX_GROUPS;
   p.ctas_done = res->d_cnt + slot;
   p.err_flag = res->d_cnt + res->n_slots;
+  p.stall_tile = ~0u;
 }
 
 // host_source: the chunk is read from mapped host memory; plain loads are used for that.
@@ -642,6 +643,11 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
   }
   uint32_t admitted = 0, submitted = 0, reaped = 0, cur_piece = 0;
   uint32_t live[BSR_MAX_RANKS] = {};
+  Inject inj;
+  {
+    std::lock_guard<std::mutex> lk(c->mu);
+    inj = c->inject;
+  }
   bool stop = false;  // a failure was seen: admit and submit nothing more, drain
 
   auto first_error = [&](int code) {
@@ -777,6 +783,10 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
       p.one.chunk = i;
       p.one.rank = r;
       for (uint32_t g = 0; g < c->G; ++g) p.one.expect[g] = o.ck[g];
+      if (inj.kind == BSR_INJECT_KERNEL_WAIT && inj.rank == r && inj.chunk == i) {
+        p.stall_tile = 0;            // the first tile of this launch is never loaded ...
+        p.wait_ns = 50ull * 1000000;  // ... and every wait in the kernel gives up after 50 ms
+      }
       const int lrc = launch_install(c, p, stream, sd, direct && o.loc == BSR_LOC_HOST);
       e = cudaEventRecord(res->ev_inst[k], stream);
       if (lrc != BSR_OK || e != cudaSuccess) {
@@ -1462,7 +1472,7 @@ int bsr_reset_stats(bsr_ctx *c) {
 
 int bsr_test_inject(bsr_ctx *c, int kind, uint32_t rank, uint32_t group, uint32_t chunk,
                     uint64_t seed) {
-  if (!c || kind < BSR_INJECT_NONE || kind > BSR_INJECT_FILL_STALL) return BSR_ERR_INVALID;
+  if (!c || kind < BSR_INJECT_NONE || kind > BSR_INJECT_KERNEL_WAIT) return BSR_ERR_INVALID;
   std::lock_guard<std::mutex> lk(c->mu);
   c->inject.kind = kind;
   c->inject.rank = rank;

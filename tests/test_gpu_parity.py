@@ -309,3 +309,26 @@ def test_direct_install_from_pinned_slots_matches_oracle(layout_name, R, N, W):
         gpu.B.bsr_test_inject(gpu.ctx, gpu.B.BSR_INJECT_CORRUPT_SLOT, r, g, i, frac)
         assert gpu.restore() == gpu.B.BSR_ERR_CHECKSUM
         assert gpu.commit() == 0 and (gpu.bitmap(N) == 0).all()
+
+
+# ---------------------------------------------------------------- a wait inside the kernel runs out
+@pytest.mark.parametrize("layout_name", ["tiny", "baseline"])
+def test_bounded_wait_inside_the_install_kernel_reports_timeout_and_context_survives(layout_name):
+    """One tile of one launch is never loaded (host-armed hook) and the kernel's waits are bounded at
+    50 ms: they expire, the kernel raises its error flag, drains its copies in flight and returns.
+    Nothing faults or hangs; the restore fails closed and the next one succeeds."""
+    layout = {"tiny": synth.tiny_layout, "baseline": synth.baseline_layout}[layout_name]()
+    R, N, W = 2, 6, 4
+    case = Case(layout, R, N, seed=1100)
+    ora = run_oracle(case, W)
+    with GpuSide(case, W) as gpu:
+        B = gpu.B
+        rc, keys, bm, n_hit = gpu.probe()
+        gpu.request(keys, n_hit)
+        assert B.bsr_test_inject(gpu.ctx, B.BSR_INJECT_KERNEL_WAIT, 1, 0, 3, 0) == B.BSR_OK
+        assert gpu.restore() == B.BSR_ERR_TIMEOUT
+        assert "bounded wait" in B.bsr_last_error(gpu.ctx)
+        assert gpu.commit() == 0 and (gpu.bitmap(N) == 0).all()
+        B.bsr_reset_stats(gpu.ctx)
+        assert gpu.restore() == B.BSR_OK                      # one shot: the context is intact
+        _check_success(case, W, gpu, ora, N)
