@@ -262,7 +262,8 @@ def run_gpu(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    layout = synth.baseline_layout()
+    layout = {"baseline": synth.baseline_layout, "hetero": synth.hetero_layout,
+              "mtp_on": synth.mtp_on_layout}[args.layout]()
     R, N, W = WORKLOAD["n_ranks"], args.chunks or WORKLOAD["n_chunks"], WORKLOAD["W"]
     chunk = layout.chunk_bytes
     seed = synth.MASTER_SEED + rank
@@ -429,6 +430,8 @@ def main():
     ap.add_argument("--load-concurrency", type=int, default=0, help="fill threads (0 = auto)")
     ap.add_argument("--depth", type=int, default=4)
     ap.add_argument("--variant", type=int, default=0, help="install kernel: 0 auto, 1 vector, 2 bulk copy")
+    ap.add_argument("--layout", default="baseline", choices=["baseline", "hetero", "mtp_on"],
+                    help="registration geometry (the contract line is the baseline one)")
     ap.add_argument("--chunks", type=int, default=0, help="prefix length in chunks (default: the workload's 128)")
     ap.add_argument("--direct", action="store_true", help="e2e arm: staging-free install (kernel reads the pinned slots)")
     ap.add_argument("--sweep", action="store_true", help="e2e GB/s vs W and vs fill concurrency (long prefixes)")

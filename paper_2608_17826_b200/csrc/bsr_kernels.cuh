@@ -1,7 +1,7 @@
 // Device code of the BSR library (sm_100a): probe, install (verify + scatter), scrub.
 //
-// Pure data movement and 64-bit integer sums: no tensor cores.  Every byte has one reader, so no
-// cluster multicast is used anywhere; bulk copies are plain per-CTA 1-D copies.
+// Pure data movement and 64-bit integer sums: no tensor cores.  Every byte has exactly one reader,
+// so every bulk copy is a plain 1-D copy into the issuing CTA's own shared memory.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -205,7 +205,7 @@ bsr_install_vec_kernel(const __grid_constant__ BsrInstallParams p) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// install, bulk variant: the copy engine of each SM (1-D bulk async copies, no multicast) moves the
+// install, bulk variant: the copy engine of each SM (1-D bulk async copies, one CTA each) moves the
 // tiles global -> shared -> global through a ring of shared-memory stages; a producer warp computes
 // addresses and issues the loads, a store warp issues the stores, and four warps sum the tile from
 // shared memory while its store is in flight.
