@@ -36,7 +36,7 @@ from paper_2608_17826_b200 import multi, synth  # noqa: E402
 WORKLOAD = dict(name="32768-token prefix, 128 chunks x 16,408,576 B, 2 rank slices, W=32, "
                      "baseline 2-group/99-tensor layout, 64-token blocks",
                 n_chunks=128, n_ranks=2, W=32)
-NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = 1.957  # profiles/install_bulk_kernel_64chunk_launch.md
+NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = 1.957  # ncu capture of the install kernel, summarised under profiles/
 METRIC, UNIT = "restore GB/s (all rank slices; per-rank = value / rank slices)", "GB/s"
 
 

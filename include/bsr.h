@@ -106,7 +106,7 @@ typedef struct bsr_tensor_desc {
 
 typedef struct bsr_stats {
   uint64_t peak_staging_bytes[BSR_MAX_RANKS];   /* max over time of live slots x slot bytes (Eq. 1) */
-  uint64_t ring_bytes_allocated[BSR_MAX_RANKS]; /* pinned ring size: W x slot bytes                  */
+  uint64_t ring_bytes_allocated[BSR_MAX_RANKS]; /* pinned pool: W (or budget B) x slot bytes         */
   uint64_t bytes_filled[BSR_MAX_RANKS];         /* tier -> slot                                      */
   uint64_t bytes_h2d[BSR_MAX_RANKS];            /* slot -> device staging                            */
   uint64_t bytes_installed[BSR_MAX_RANKS];      /* verified and scattered                            */
@@ -206,10 +206,11 @@ int bsr_req_release(bsr_ctx *ctx, bsr_req *req);
 /* ---- restore (Section 2 "Bounded installation", Section 3 "Install locally") -------------- */
 
 /* Installs the advertised prefix of every rank.  Chunk i of rank r is copied from the tier into
- * pinned slot i mod W of r's ring (at most W slots live per rank, a slot is live from before its
- * fill until its install has been observed complete), copied to a device staging buffer on the
- * library's copy stream, then verified and scattered through the block tables by the install
- * kernel on `cuda_stream` (a cudaStream_t, or NULL for a stream owned by the library).  The first
+ * a free pinned slot of r's pool (this restore holds at most W slots per rank; a slot is live from
+ * its admission, before the fill, until its install has been observed complete), copied to a
+ * device staging buffer on the library's copy stream, then verified and scattered through the
+ * block tables by the install kernel on `cuda_stream` (a cudaStream_t, or NULL for a stream owned
+ * by the library).  Objects that live in device memory are installed in place.  The first
  * missing key, checksum mismatch, transfer error or deadline overrun stops admission, drains what
  * is in flight, invalidates the whole request and is returned.  Blocking; on return no slot is
  * live and every kernel of the call has finished.

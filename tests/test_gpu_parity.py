@@ -311,6 +311,26 @@ def test_direct_install_from_pinned_slots_matches_oracle(layout_name, R, N, W):
         assert gpu.commit() == 0 and (gpu.bitmap(N) == 0).all()
 
 
+# ---------------------------------------------------------------- limits of the interface
+def test_maximum_ranks_groups_and_extreme_block_sizes():
+    """8 rank slices x 8 allocator groups (the interface maxima), block sizes from 2 tokens (128 blocks
+    per chunk) to 256 tokens (one block per chunk), tensors of 16 B/token (16-byte runs split nowhere)."""
+    blocks = [2, 4, 8, 16, 32, 64, 128, 256]
+    tensors = [(g, e) for g, e in zip(range(8), [16, 32, 16, 48, 16, 64, 16, 80])] + [(7, 16)]
+    layout = synth.Layout("limits", blocks, sorted(tensors))
+    R, N, W = 8, 5, 2
+    case = Case(layout, R, N, seed=1200)
+    ora = run_oracle(case, W)
+    assert ora["status"] == O.OK
+    for cfg in (dict(), dict(install_variant=1), dict(direct_install=True), dict(location=1)):
+        with GpuSide(case, W, **cfg) as gpu:
+            rc, keys, bm, n_hit = gpu.probe()
+            assert n_hit == N
+            gpu.request(keys, n_hit)
+            assert gpu.restore() == gpu.B.BSR_OK, gpu.B.bsr_last_error(gpu.ctx)
+            _check_success(case, W, gpu, ora, N)
+
+
 # ---------------------------------------------------------------- a wait inside the kernel runs out
 @pytest.mark.parametrize("layout_name", ["tiny", "baseline"])
 def test_bounded_wait_inside_the_install_kernel_reports_timeout_and_context_survives(layout_name):
