@@ -391,7 +391,8 @@ def run_sweep(args):
     R, P, seed = 2, 67, synth.MASTER_SEED
     objs = {(r, j): synth.chunk_payload(layout, r, j, seed=seed).copy() for r in range(R) for j in range(P)}
     h2d = measure_h2d(torch, dev, layout.chunk_bytes)
-    plan = [(N, W, 0) for N in (512, 1024) for W in (8, 16, 32, 64)] + [(512, 32, lc) for lc in (1, 2, 4, 8, 16)]
+    plan = ([(N, W, 0) for N in (512, 1024) for W in (8, 16, 32, 64)] + [(2048, 32, 0)] +
+            [(512, 32, lc) for lc in (1, 2, 4, 8, 16)])
     for N, W, lc in plan:
         tok = synth.tokens(N * 256, seed=seed + N)
         payload = {(r, i): objs[(r, i % P)] for r in range(R) for i in range(N)}

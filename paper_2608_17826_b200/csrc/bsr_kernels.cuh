@@ -9,7 +9,9 @@
 
 #define BSR_K_MAX_GROUPS 8
 #define BSR_K_MAX_BATCH 256       // chunk descriptors per install launch
+#ifndef BSR_K_TILE_MAX
 #define BSR_K_TILE_MAX 16384u     // largest tile in bytes (one bulk-copy stage)
+#endif
 #define BSR_K_PHI 0x9E3779B97F4A7C15ull
 
 // ---------------------------------------------------------------------------------------------
@@ -218,7 +220,12 @@ bsr_install_vec_kernel(const __grid_constant__ BsrInstallParams p) {
 // Every wait is bounded by a wall-clock deadline; a wait that gives up raises *err_flag, the CTA
 // stops issuing work, drains what it has in flight and leaves through the common exit.
 // ---------------------------------------------------------------------------------------------
+#ifndef BSR_K_BULK_STAGES
 #define BSR_K_BULK_STAGES 6
+#endif
+#ifndef BSR_K_BULK_CTAS_PER_SM
+#define BSR_K_BULK_CTAS_PER_SM 2  // 2 x 6 stages x 16 KiB = 192 KiB of the SM's shared memory
+#endif
 #define BSR_K_BULK_CONSUMER_WARPS 4
 #define BSR_K_BULK_THREADS (32 * (2 + BSR_K_BULK_CONSUMER_WARPS))
 #define BSR_K_BULK_STORE_LAG 2  // stores whose shared-memory reads may still be pending

@@ -293,7 +293,7 @@ int launch_install(bsr_ctx *c, const BsrInstallParams &p, cudaStream_t s, StatDe
                    bool host_source = false) {
   const uint64_t total = (uint64_t)p.n_chunks * p.n_tiles;
   if (c->cfg.install_variant != BSR_INSTALL_VECTOR && !host_source) {  // AUTO = bulk copies
-    const uint64_t want = (uint64_t)kSmCount * 2;  // two CTAs of 6 x 16 KiB stages per SM
+    const uint64_t want = (uint64_t)kSmCount * BSR_K_BULK_CTAS_PER_SM;  // persistent: one wave
     bsr_install_bulk_kernel<<<(uint32_t)(total < want ? total : want), BSR_K_BULK_THREADS,
                               BSR_K_BULK_SMEM, s>>>(p);
   } else {
