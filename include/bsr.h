@@ -17,7 +17,8 @@
  *     the context's GPU.  The library never frees memory it did not allocate.
  *   - Handles (bsr_ctx, bsr_req) are opaque.  A context is bound to one GPU.  Calls on one context
  *     may come from any thread; restores on one context are serialised by a context-wide lock
- *     (Section 3 "Install locally": concurrent requests must not multiply the staging budget).
+ *     (Section 3 "Install locally": concurrent requests must not multiply the staging budget)
+ *     unless bsr_config.budget_slots sets a shared admission budget for concurrent restores.
  *   - All integer arithmetic of the method is unsigned, modulo 2^64.
  *
  * Functions the paper leaves open and this library defines (documented at each call): the chunk
@@ -241,6 +242,19 @@ int bsr_req_checksums(bsr_ctx *ctx, bsr_req *req, uint64_t *out, size_t count);
 
 int bsr_get_stats(bsr_ctx *ctx, bsr_stats *out);
 int bsr_reset_stats(bsr_ctx *ctx);
+
+/* Timeline of one chunk of one rank through the window: nanoseconds since the restore started. */
+typedef struct bsr_trace_rec {
+  uint32_t chunk, rank, slot, reserved;
+  uint64_t t_admit_ns;  /* a slot was reserved for the chunk (it becomes live)                  */
+  uint64_t t_filled_ns; /* the last piece of the tier object landed in the slot                 */
+  uint64_t t_submit_ns; /* its copies and its install launch were queued                        */
+  uint64_t t_done_ns;   /* its install was observed complete and the slot released; 0 = never   */
+} bsr_trace_rec;
+
+/* Copies the timeline of the most recent restore that went through the slot pool (one record per
+ * admitted (chunk, rank), in admission order) into out[capacity]; *count = records available. */
+int bsr_get_trace(bsr_ctx *ctx, bsr_trace_rec *out, size_t capacity, size_t *count);
 
 /* ---- host-side failure injection (tests) -------------------------------------------------- */
 

@@ -34,6 +34,7 @@ EXPORTS = [
     "bsr_req_checksums", "bsr_get_stats", "bsr_reset_stats", "bsr_test_inject",
     "bsr_probe_keys_noalloc", "bsr_tier_put_at", "bsr_tier_remove_at", "bsr_tier_set_available",
     "bsr_probe_request", "bsr_req_bind", "bsr_request_done", "bsr_request_is_force_local",
+    "bsr_get_trace",
 ]
 BSR_MAX_TIERS = 4
 BSR_NOALLOC_MAX_CHUNKS = 8192
@@ -66,6 +67,12 @@ class bsr_stats(C.Structure):
                 ("h2d_copies", C.c_uint64), ("install_launches", C.c_uint64),
                 ("bytes_restored_by_tier", C.c_uint64 * 4),
                 ("install_kernel_ms", C.c_double), ("last_restore_ms", C.c_double)]
+
+
+class bsr_trace_rec(C.Structure):
+    _fields_ = [("chunk", C.c_uint32), ("rank", C.c_uint32), ("slot", C.c_uint32), ("reserved", C.c_uint32),
+                ("t_admit_ns", C.c_uint64), ("t_filled_ns", C.c_uint64), ("t_submit_ns", C.c_uint64),
+                ("t_done_ns", C.c_uint64)]
 
 
 def _load() -> C.CDLL:
@@ -102,6 +109,7 @@ def _load() -> C.CDLL:
         "bsr_req_bind": [vp, vp, u64, u32],
         "bsr_request_done": [vp, u64],
         "bsr_request_is_force_local": [vp, u64, C.POINTER(i32)],
+        "bsr_get_trace": [vp, vp, C.c_size_t, C.POINTER(C.c_size_t)],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -285,3 +293,13 @@ def bsr_request_is_force_local(ctx, request_id: int):
     out = C.c_int(0)
     rc = lib.bsr_request_is_force_local(ctx, int(request_id), C.byref(out))
     return rc, bool(out.value)
+
+
+def bsr_get_trace(ctx, capacity: int = 1 << 16):
+    """Returns (rc, numpy structured array) with the timeline of the last restore through the slot pool."""
+    dt = np.dtype([("chunk", "<u4"), ("rank", "<u4"), ("slot", "<u4"), ("reserved", "<u4"),
+                   ("t_admit_ns", "<u8"), ("t_filled_ns", "<u8"), ("t_submit_ns", "<u8"), ("t_done_ns", "<u8")])
+    out = np.zeros(capacity, dtype=dt)
+    n = C.c_size_t(0)
+    rc = lib.bsr_get_trace(ctx, out.ctypes.data, capacity, C.byref(n))
+    return rc, out[: min(n.value, capacity)]

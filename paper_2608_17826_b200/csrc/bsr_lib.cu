@@ -89,6 +89,9 @@ struct Job {
   std::unique_ptr<std::atomic<int>[]> state;  // per piece: 0 pending, 1 ready, <0 error
   std::vector<TierObj> objs;                  // per (chunk, rank)
   std::vector<uint32_t> slot;                 // per (chunk, rank): slot of the rank's pool
+  std::vector<uint64_t> t_piece;              // per piece: ns since restore start when its fill ended
+  std::vector<bsr_trace_rec> trace;           // per (chunk, rank)
+  Clock::time_point t0;
   std::atomic<bool> abort{false};
   uint32_t fill_admitted = 0, fill_next = 0, fill_active = 0;  // guarded by fill_mu
 };
@@ -144,6 +147,7 @@ struct bsr_ctx {
   std::unordered_set<uint64_t> force_local;  // request ids whose next probe must report zero
   Inject inject;
   bsr_stats st{};
+  std::vector<bsr_trace_rec> last_trace;  // timeline of the last restore through the slot pool
 
   // context-level stream and scratch for probe, store-path checksums, scrub (aux_mu)
   cudaStream_t copy_stream = nullptr, own_stream = nullptr;
@@ -487,6 +491,7 @@ void filler_main(bsr_ctx *c) {
       }
     }
     if (piece == 0) job->objs[s] = obj;
+    job->t_piece[t] = (uint64_t)std::chrono::duration_cast<std::chrono::nanoseconds>(Clock::now() - job->t0).count();
     job->state[t].store(state, std::memory_order_release);
     {
       std::lock_guard<std::mutex> lk(c->fill_mu);
@@ -637,6 +642,12 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
   for (size_t k = 0; k < (size_t)total * P; ++k) job.state[k].store(0, std::memory_order_relaxed);
   job.objs.resize(total);
   job.slot.assign(total, 0);
+  job.t_piece.assign((size_t)total * P, 0);
+  job.trace.assign(total, bsr_trace_rec{});
+  job.t0 = Clock::now();
+  auto now_ns = [&] {
+    return (uint64_t)std::chrono::duration_cast<std::chrono::nanoseconds>(Clock::now() - job.t0).count();
+  };
   {
     std::lock_guard<std::mutex> lk(c->fill_mu);
     c->jobs.push_back(&job);
@@ -680,6 +691,10 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
           if (bytes > c->st.peak_staging_bytes[r]) c->st.peak_staging_bytes[r] = bytes;
         }
         if (i % W == 0 && r == 0) sd.windows++;
+        job.trace[admitted].chunk = i;
+        job.trace[admitted].rank = r;
+        job.trace[admitted].slot = job.slot[admitted];
+        job.trace[admitted].t_admit_ns = now_ns();
         live[r]++;
         ++admitted;
         ++n_new;
@@ -714,6 +729,7 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
       }
       const int h = harvest(c, q, r, i, sd);
       if (h != BSR_OK) first_error(h);
+      job.trace[reaped].t_done_ns = now_ns();
       release_slot(reaped);
       live[r]--;
       ++reaped;
@@ -793,6 +809,10 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
         first_error(lrc != BSR_OK ? lrc : fail(c, BSR_ERR_CUDA, "record: %s", cudaGetErrorString(e)));
         break;
       }
+      for (uint32_t pc = 0; pc < P; ++pc)
+        if (job.t_piece[(size_t)submitted * P + pc] > job.trace[submitted].t_filled_ns)
+          job.trace[submitted].t_filled_ns = job.t_piece[(size_t)submitted * P + pc];
+      job.trace[submitted].t_submit_ns = now_ns();
       ++submitted;
       cur_piece = 0;
       progress = true;
@@ -826,6 +846,11 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
   }
   // slots admitted but never installed go back to the pool
   for (uint32_t s = reaped; s < admitted; ++s) release_slot(s);
+  {
+    std::lock_guard<std::mutex> lk(c->mu);
+    job.trace.resize(admitted);
+    c->last_trace.swap(job.trace);
+  }
   return rc;
 }
 
@@ -1454,6 +1479,15 @@ int bsr_get_stats(bsr_ctx *c, bsr_stats *out) {
   std::lock_guard<std::mutex> pl(c->pool_mu);  // peak_staging_bytes is written under pool_mu
   std::lock_guard<std::mutex> lk(c->mu);
   *out = c->st;
+  return BSR_OK;
+}
+
+int bsr_get_trace(bsr_ctx *c, bsr_trace_rec *out, size_t capacity, size_t *count) {
+  if (!c || !count || (!out && capacity)) return BSR_ERR_INVALID;
+  std::lock_guard<std::mutex> lk(c->mu);
+  *count = c->last_trace.size();
+  const size_t n = *count < capacity ? *count : capacity;
+  if (n) memcpy(out, c->last_trace.data(), n * sizeof(bsr_trace_rec));
   return BSR_OK;
 }
 

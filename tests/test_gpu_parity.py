@@ -311,6 +311,40 @@ def test_direct_install_from_pinned_slots_matches_oracle(layout_name, R, N, W):
         assert gpu.commit() == 0 and (gpu.bitmap(N) == 0).all()
 
 
+# ---------------------------------------------------------------- the timeline shows Eq. 3
+@pytest.mark.parametrize("N,W,depth", [(40, 4, 2), (25, 8, 4), (9, 16, 1)])
+def test_timeline_of_a_restore_never_has_more_than_w_live_chunks_per_rank(N, W, depth):
+    layout = synth.Layout("mid", [64, 16], [(0, 1024), (1, 256)])      # 320 KiB chunks
+    R = 2
+    case = Case(layout, R, N, seed=1300 + N)
+    with GpuSide(case, W, dev_staging_depth=depth) as gpu:
+        B = gpu.B
+        rc, keys, bm, n_hit = gpu.probe()
+        gpu.request(keys, n_hit)
+        assert gpu.restore() == B.BSR_OK
+        rc, tr = B.bsr_get_trace(gpu.ctx)
+        assert rc == B.BSR_OK and len(tr) == N * R
+        assert sorted((int(t["chunk"]), int(t["rank"])) for t in tr) == [(i, r) for i in range(N) for r in range(R)]
+        assert (tr["t_admit_ns"] <= tr["t_filled_ns"]).all() and (tr["t_filled_ns"] <= tr["t_submit_ns"]).all()
+        assert (tr["t_submit_ns"] < tr["t_done_ns"]).all() and (tr["slot"] < W).all()
+        for r in range(R):
+            t = tr[tr["rank"] == r]
+            # sweep the admit (+1) and release (-1) instants: live slots of the rank never exceed W (Eq. 3) ...
+            ev = sorted([(int(x), 1) for x in t["t_admit_ns"]] + [(int(x), -1) for x in t["t_done_ns"]],
+                        key=lambda e: (e[0], e[1]))
+            live = peak = 0
+            for _, d in ev:
+                live += d
+                peak = max(peak, live)
+            assert peak == min(N, W)                                    # ... and do reach it
+            # no slot is handed to a second chunk while its previous chunk is still live
+            for s in set(int(x) for x in t["slot"]):
+                u = t[t["slot"] == s]
+                u = u[np.argsort(u["t_admit_ns"])]
+                assert (u["t_done_ns"][:-1] <= u["t_admit_ns"][1:]).all()
+        assert gpu.stats().peak_staging_bytes[0] == min(N, W) * case.reg.slot_bytes
+
+
 # ---------------------------------------------------------------- limits of the interface
 def test_maximum_ranks_groups_and_extreme_block_sizes():
     """8 rank slices x 8 allocator groups (the interface maxima), block sizes from 2 tokens (128 blocks
