@@ -77,6 +77,12 @@ class bsr_trace_rec(C.Structure):
 
 def _load() -> C.CDLL:
     if not os.path.exists(LIB_PATH):
+        try:  # a fresh checkout: compile once with nvcc, in-tree
+            from . import build as _build
+            _build.build()
+        except Exception as exc:  # noqa: BLE001 - reported below, never hidden behind a fallback
+            raise ImportError(f"{LIB_PATH} is missing and could not be built: {exc}") from exc
+    if not os.path.exists(LIB_PATH):
         raise ImportError(
             f"{LIB_PATH} is missing: build it with `python -m paper_2608_17826_b200.build` "
             "(needs nvcc). The BSR path has no CPU fallback.")
