@@ -135,6 +135,30 @@ def test_a_failing_request_fails_alone_under_a_budget():
         c.close()
 
 
+def test_four_concurrent_restores_one_failing():
+    c = TwoRequests([70, 55, 64, 40], 4, 10, corrupt=(2, 1, 33), load_concurrency=6)
+    try:
+        B = c.B
+        statuses = c.run_gpu_concurrently()
+        c.compare(statuses)
+        assert statuses == [B.BSR_OK, B.BSR_OK, B.BSR_ERR_CHECKSUM, B.BSR_OK]
+        for k in (0, 1, 3):                                          # the healthy ones are bit-exact
+            oq = c.oreqs[k]
+            for r in range(R):
+                for l, (g, _) in enumerate(c.layout.tensors):
+                    used = oq.block_tables[r][g]
+                    assert np.array_equal(c.gpaged[r][l].cpu().numpy()[used], c.opaged[r][l][used])
+        st = B.bsr_get_stats(c.ctx)[1]
+        slot = c.reg.slot_bytes
+        assert 4 * slot <= max(st.peak_staging_bytes[:R]) <= 10 * slot
+        # after the storm every slot is back: a single restore can again hold W and no more
+        B.bsr_reset_stats(c.ctx)
+        assert B.bsr_restore(c.ctx, c.greqs[0], None) == B.BSR_OK
+        assert B.bsr_get_stats(c.ctx)[1].peak_staging_bytes[0] == 4 * slot
+    finally:
+        c.close()
+
+
 def test_sequential_restores_with_a_budget_behave_like_the_locked_mode():
     c = TwoRequests([40, 30], 8, 20)
     try:

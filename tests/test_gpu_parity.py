@@ -311,6 +311,31 @@ def test_direct_install_from_pinned_slots_matches_oracle(layout_name, R, N, W):
         assert gpu.commit() == 0 and (gpu.bitmap(N) == 0).all()
 
 
+# ---------------------------------------------------------------- many pipeline shapes
+def test_many_pipeline_shapes_give_the_same_bytes():
+    """Seeded sweep over W, fill threads, staging depth, install path and ranks on one small case:
+    ordering bugs in the slot pool / copy / install pipeline would show as a byte or bitmap mismatch."""
+    rng = np.random.default_rng(20260817)
+    layout = synth.Layout("mid", [64, 16], [(0, 1024), (0, 48), (1, 256)])
+    oracles = {}
+    for trial in range(16):
+        R = int(rng.integers(1, 4))
+        N = int(rng.integers(1, 40))
+        W = int(rng.choice([1, 2, 3, 5, 8, 64]))
+        cfg = dict(load_concurrency=int(rng.choice([1, 2, 4, 8])), dev_staging_depth=int(rng.choice([1, 2, 4, 7])),
+                   install_variant=int(rng.choice([1, 2])), direct_install=bool(rng.integers(0, 2)))
+        case = Case(layout, R, N, seed=1400 + trial)
+        ora = run_oracle(case, W)
+        with GpuSide(case, W, **cfg) as gpu:
+            rc, keys, bm, n_hit = gpu.probe(tok_on_device=bool(trial % 2))
+            assert rc == gpu.B.BSR_OK and n_hit == N, (trial, cfg)
+            gpu.request(keys, n_hit)
+            for _ in range(2):
+                gpu.B.bsr_reset_stats(gpu.ctx)
+                assert gpu.restore() == gpu.B.BSR_OK, (trial, cfg, gpu.B.bsr_last_error(gpu.ctx))
+                _check_success(case, W, gpu, ora, N)
+
+
 # ---------------------------------------------------------------- the timeline shows Eq. 3
 @pytest.mark.parametrize("N,W,depth", [(40, 4, 2), (25, 8, 4), (9, 16, 1)])
 def test_timeline_of_a_restore_never_has_more_than_w_live_chunks_per_rank(N, W, depth):
