@@ -40,6 +40,9 @@ constexpr int kInstallUnroll = 4;
 constexpr int kLaunchSlots = 8;  // scratch sets for batched install launches in flight per restore
 constexpr uint32_t kSmCount = 148;
 constexpr uint64_t kPieceBytes = 8ull << 20;  // fill and host-to-device copy granularity
+#ifndef BSR_RING_ALLOC_FLAGS
+#define BSR_RING_ALLOC_FLAGS cudaHostAllocMapped
+#endif
 
 struct TierObj {
   const uint8_t *data;
@@ -508,7 +511,7 @@ int ensure_ring(bsr_ctx *c) {
   if (c->ring_ready.load(std::memory_order_acquire)) return BSR_OK;
   const uint32_t R = c->cfg.n_ranks, B = c->budget;
   for (uint32_t r = 0; r < R; ++r) {
-    if (cudaHostAlloc((void **)&c->ring[r], (size_t)B * c->slot_bytes, cudaHostAllocMapped) !=
+    if (cudaHostAlloc((void **)&c->ring[r], (size_t)B * c->slot_bytes, BSR_RING_ALLOC_FLAGS) !=
             cudaSuccess ||
         cudaHostGetDevicePointer((void **)&c->ring_dev[r], c->ring[r], 0) != cudaSuccess) {
       cudaGetLastError();
