@@ -125,9 +125,10 @@ typedef struct bsr_stats {
 
 /* ---- context ------------------------------------------------------------------------------- */
 
-/* Creates a context on cfg->device.  Allocates nothing proportional to a prefix; the pinned ring
- * (W slots per rank) and the device staging buffers are allocated at the first restore, when the
- * chunk size is known.  Errors: INVALID (W = 0, ranks out of range, chunk_tokens != 256), CUDA. */
+/* Creates a context on cfg->device.  Allocates nothing proportional to a prefix; the pinned slot
+ * pool (W slots per rank, or B with an admission budget) and the device staging buffers are
+ * allocated at the first restore, when the chunk size is known.
+ * Errors: INVALID (W = 0, ranks out of range, chunk_tokens != 256), CUDA (no usable device). */
 int bsr_ctx_create(const bsr_config *cfg, bsr_ctx **out);
 
 /* Destroys the context, its ring, staging, index and any request still alive. */
@@ -202,6 +203,8 @@ int bsr_probe(bsr_ctx *ctx, const int32_t *tok, size_t n_tok, int tok_on_device,
 int bsr_req_create(bsr_ctx *ctx, const uint64_t *keys, uint32_t n_adv_chunks,
                    const int32_t *const *block_tables, bsr_req **out);
 
+/* Frees the request and its device-side tables (waits for a call in flight on it).  Nothing the
+ * caller passed at creation is referenced afterwards: keys and tables were copied. */
 int bsr_req_release(bsr_ctx *ctx, bsr_req *req);
 
 /* ---- restore (Section 2 "Bounded installation", Section 3 "Install locally") -------------- */
@@ -240,6 +243,9 @@ int bsr_req_bitmap(bsr_ctx *ctx, bsr_req *req, uint64_t *out, size_t words);
 /* Checksums the install kernel computed, out[(r*G + g) * n_adv + i]; 0 where not installed. */
 int bsr_req_checksums(bsr_ctx *ctx, bsr_req *req, uint64_t *out, size_t count);
 
+/* Copies the context's counters (Eq. 1 peak, byte counters of every stage, windows, launches).
+ * bsr_reset_stats zeroes them, keeping only the sizes of what stays allocated (slot_bytes,
+ * ring_bytes_allocated, dev_aux_bytes). */
 int bsr_get_stats(bsr_ctx *ctx, bsr_stats *out);
 int bsr_reset_stats(bsr_ctx *ctx);
 
