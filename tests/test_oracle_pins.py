@@ -327,6 +327,26 @@ def test_commit_truth_table_every_subset_of_failing_components():
             assert 0 < max(st.peak_staging_bytes) <= W * reg.slot_bytes
 
 
+def test_commit_is_the_conjunction_of_eq6_on_every_bit_pattern():
+    """Eq. 6 on the predicate itself: for every pattern of the q_{r,g} bits (one chunk), commit exposes
+    the prefix only when all are set and a restore completed; one missing bit of any rank or group is zero."""
+    layout = synth.tiny_layout()
+    R, G = 2, layout.n_groups
+    for mask in range(1 << (R * G)):
+        reg, tok, tiers, keys, tables, paged, payload, pools = _build_case(layout, R, 1, seed=62)
+        req = O.Request(keys[:1], tables, R, G)
+        for bit, (r, g) in enumerate(itertools.product(range(R), range(G))):
+            req.valid[r, g, 0] = bool(mask >> bit & 1)
+        req.restored = True
+        assert O.commit(reg, req, paged) == (1 if mask == (1 << (R * G)) - 1 else 0)
+    # all bits set but no completed restore, or a failed one: nothing is exposed
+    for restored, failed in ((False, False), (True, True)):
+        req = O.Request(keys[:1], tables, R, G)
+        req.valid[:] = True
+        req.restored, req.failed = restored, failed
+        assert O.commit(reg, req, paged) == 0
+
+
 def test_failure_cases_are_fail_closed_and_scrub_zeroes_only_request_blocks():
     layout = synth.tiny_layout()
     R, N, W = 2, 9, 3
