@@ -363,7 +363,9 @@ def run_gpu(args):
         "peak_staging_bytes_per_rank": peak_staging, "staging_law_bytes": W * slot,
         "staging_residual_bytes": [p - W * slot for p in peak_staging],
         "gpu_launches": launches,
-        "roofline": {"bound": "hbm", "kernel": "bsr_install_*_kernel", "achieved": achieved,
+        "roofline": {"bound": "hbm",
+                     "kernel": "bsr_install_vec_kernel" if args.variant == 1 else "bsr_install_bulk_kernel",
+                     "achieved": achieved,
                      "peak": hbm_peak, "unit": "GB/s", "frac": (achieved / hbm_peak) if achieved else None,
                      "traffic": traffic, "peak_source": peak_src,
                      "launches": k_launches, "avg_launch_ms": k_ms,
