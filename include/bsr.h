@@ -131,11 +131,13 @@ typedef struct bsr_stats {
  * Errors: INVALID (W = 0, ranks out of range, chunk_tokens != 256), CUDA (no usable device). */
 int bsr_ctx_create(const bsr_config *cfg, bsr_ctx **out);
 
-/* Destroys the context, its ring, staging, index and any request still alive. */
+/* Destroys the context, its slot pool, staging and index.  Release every request of the context
+ * first (bsr_req_release) and let no call be in flight on it. */
 int bsr_ctx_destroy(bsr_ctx *ctx);
 
 /* Text of the last CUDA or argument error seen by this context (never NULL; valid until the next
- * failing call on the context). */
+ * failing call on the context; read it from the thread that saw the failing call, with no other
+ * call running on the context). */
 const char *bsr_last_error(bsr_ctx *ctx);
 
 /* ---- registration (Section 4: registered tensors in allocator groups, per TP rank) -------- */

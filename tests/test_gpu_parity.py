@@ -56,6 +56,27 @@ def test_probe_keys_bitmap_prefix(N, tail, on_device):
         assert rc == gpu.B.BSR_OK and nh2 == 0 and not np.array_equal(k2, keys)
 
 
+def test_probe_sixteen_million_tokens_and_scratch_regrowth():
+    """65,539 chunks: many passes of the key chain through its shared-memory tile, scratch grown
+    twice (a short probe first), and the boundary chunk counts of the digest grid."""
+    import torch
+    from paper_2608_17826_b200 import binding as B
+    rc, ctx = B.bsr_ctx_create(4, 1, reg_id=77)
+    assert rc == B.BSR_OK
+    try:
+        for n_chunks in (3, 65539, 2047):
+            tok = synth.tokens(n_chunks * 256 + 5, seed=1500 + n_chunks)
+            want = O.prefix_keys(O.chunk_digests(tok, 0xFEED), 0xFEED, 77)
+            rc, keys, bm, n_hit = B.bsr_probe(ctx, tok, len(tok), 0xFEED, False)
+            assert rc == B.BSR_OK and n_hit == 0 and np.array_equal(keys, want) and not bm.any()
+            d_tok = torch.from_numpy(tok).cuda()
+            torch.cuda.synchronize()
+            rc, keys, bm, n_hit = B.bsr_probe(ctx, d_tok.data_ptr(), len(tok), 0xFEED, True)
+            assert rc == B.BSR_OK and np.array_equal(keys, want)
+    finally:
+        B.bsr_ctx_destroy(ctx)
+
+
 def test_probe_fewer_than_one_chunk():
     case = Case(synth.tiny_layout(), 1, 1, seed=102)
     with GpuSide(case, W=2) as gpu:
