@@ -293,6 +293,20 @@ int bsr_tier_put_at(bsr_ctx *ctx, uint32_t tier, uint32_t rank, uint64_t key, co
                     size_t len, const uint64_t *group_ck, int location);
 int bsr_tier_remove_at(bsr_ctx *ctx, uint32_t tier, uint32_t rank, uint64_t key);
 
+/* Tier adapter (Section 4 "Storage-side concurrency is orthogonal": reads fill the same
+ * preallocated window objects).  For a tier whose bytes are not in addressable memory (a file,
+ * a remote store), register a fetch function and put the objects with data = NULL, BSR_LOC_HOST
+ * and their checksums.  At restore time the library calls, from its fill threads and up to
+ * load_concurrency at once,
+ *     fn(user, tier, rank, key, offset, len, dst)
+ * to deliver bytes [offset, offset + len) of the object straight into the pinned staging slot at
+ * dst (pieces of at most 8 MiB, in no particular order).  Return 0 on success; any other value
+ * fails the restore closed with BSR_ERR_TRANSFER.  fn must be thread-safe and must not call back
+ * into the context.  NULL removes the adapter. */
+typedef int (*bsr_fetch_fn)(void *user, uint32_t tier, uint32_t rank, uint64_t key, uint64_t offset,
+                            uint64_t len, void *dst);
+int bsr_tier_set_fetch(bsr_ctx *ctx, uint32_t tier, bsr_fetch_fn fn, void *user);
+
 /* Marks a tier reachable (default) or unreachable.  An unreachable tier is skipped by
  * bsr_probe_request, and a restore bound to it fails closed with BSR_ERR_TRANSFER. */
 int bsr_tier_set_available(bsr_ctx *ctx, uint32_t tier, int available);

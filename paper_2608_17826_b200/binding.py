@@ -34,8 +34,11 @@ EXPORTS = [
     "bsr_req_checksums", "bsr_get_stats", "bsr_reset_stats", "bsr_test_inject",
     "bsr_probe_keys_noalloc", "bsr_tier_put_at", "bsr_tier_remove_at", "bsr_tier_set_available",
     "bsr_probe_request", "bsr_req_bind", "bsr_request_done", "bsr_request_is_force_local",
-    "bsr_get_trace",
+    "bsr_get_trace", "bsr_tier_set_fetch",
 ]
+# int fn(void *user, uint32 tier, uint32 rank, uint64 key, uint64 offset, uint64 len, void *dst)
+BSR_FETCH_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint64, C.c_uint64,
+                           C.c_uint64, C.c_void_p)
 BSR_MAX_TIERS = 4
 BSR_NOALLOC_MAX_CHUNKS = 8192
 
@@ -116,6 +119,7 @@ def _load() -> C.CDLL:
         "bsr_request_done": [vp, u64],
         "bsr_request_is_force_local": [vp, u64, C.POINTER(i32)],
         "bsr_get_trace": [vp, vp, C.c_size_t, C.POINTER(C.c_size_t)],
+        "bsr_tier_set_fetch": [vp, u32, BSR_FETCH_FN, vp],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -299,6 +303,11 @@ def bsr_request_is_force_local(ctx, request_id: int):
     out = C.c_int(0)
     rc = lib.bsr_request_is_force_local(ctx, int(request_id), C.byref(out))
     return rc, bool(out.value)
+
+
+def bsr_tier_set_fetch(ctx, tier: int, fn, user=None) -> int:
+    """fn: a BSR_FETCH_FN instance (keep a reference to it for as long as it is registered), or None."""
+    return lib.bsr_tier_set_fetch(ctx, tier, fn if fn is not None else BSR_FETCH_FN(0), user)
 
 
 def bsr_get_trace(ctx, capacity: int = 1 << 16):

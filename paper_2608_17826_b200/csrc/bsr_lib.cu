@@ -147,6 +147,8 @@ struct bsr_ctx {
   // tiers + index (mu)
   std::unordered_map<uint64_t, TierObj> tier[BSR_MAX_TIERS][BSR_MAX_RANKS];
   bool tier_available[BSR_MAX_TIERS] = {true, true, true, true};
+  bsr_fetch_fn fetch_fn[BSR_MAX_TIERS] = {};  // tier adapters: fill a slot for objects put without data
+  void *fetch_user[BSR_MAX_TIERS] = {};
   std::unordered_set<uint64_t> force_local;  // request ids whose next probe must report zero
   Inject inject;
   bsr_stats st{};
@@ -459,6 +461,8 @@ void filler_main(bsr_ctx *c) {
     if (!job->abort.load(std::memory_order_acquire)) {
       bool found = false, tier_down = false;
       Inject inj;
+      bsr_fetch_fn fetch = nullptr;
+      void *fetch_user = nullptr;
       {
         std::lock_guard<std::mutex> g(c->mu);
         auto &index = c->tier[req->tier][r];
@@ -469,6 +473,8 @@ void filler_main(bsr_ctx *c) {
         }
         if (!c->tier_available[req->tier]) tier_down = true;
         inj = c->inject;
+        fetch = c->fetch_fn[req->tier];
+        fetch_user = c->fetch_user[req->tier];
       }
       const bool hit = inj.kind != BSR_INJECT_NONE && inj.rank == r && inj.chunk == i;
       if (tier_down) {
@@ -484,8 +490,13 @@ void filler_main(bsr_ctx *c) {
         state = BSR_ERR_TIMEOUT;
       } else if (obj.loc == BSR_LOC_HOST) {
         uint8_t *slot = c->ring[r] + (size_t)job->slot[s] * c->slot_bytes;
-        fill_copy(slot + off, obj.data + off, len);
-        if (hit && inj.kind == BSR_INJECT_CORRUPT_SLOT && inj.group < c->G) {
+        if (obj.data) {
+          fill_copy(slot + off, obj.data + off, len);
+        } else if (!fetch ||
+                   fetch(fetch_user, req->tier, r, req->keys[i], off, len, slot + off) != 0) {
+          state = BSR_ERR_TRANSFER;  // the tier adapter could not deliver the bytes
+        }
+        if (state == 1 && hit && inj.kind == BSR_INJECT_CORRUPT_SLOT && inj.group < c->G) {
           const uint64_t words = c->seg_bytes[inj.group] / 4;
           const uint64_t at = c->seg_begin[inj.group] + 4 * (inj.seed % words);
           if (at >= off && at < off + len)
@@ -1118,9 +1129,21 @@ int bsr_tier_put(bsr_ctx *c, uint32_t rank, uint64_t key, const void *data, size
 
 int bsr_tier_put_at(bsr_ctx *c, uint32_t tier, uint32_t rank, uint64_t key, const void *data,
                     size_t len, const uint64_t *group_ck, int location) {
-  if (!c || !data || tier >= BSR_MAX_TIERS) return BSR_ERR_INVALID;
+  if (!c || tier >= BSR_MAX_TIERS) return BSR_ERR_INVALID;
   if (rank >= c->cfg.n_ranks || (location != BSR_LOC_HOST && location != BSR_LOC_DEVICE))
     return fail(c, BSR_ERR_INVALID, "tier_put: bad rank or location");
+  if (!data) {
+    // an index entry without bytes: the tier's fetch adapter delivers them at restore time
+    bool adapter;
+    {
+      std::lock_guard<std::mutex> lk(c->mu);
+      adapter = c->fetch_fn[tier] != nullptr;
+    }
+    if (!adapter || !group_ck || location != BSR_LOC_HOST)
+      return fail(c, BSR_ERR_INVALID,
+                  "tier_put: an object without data needs a fetch adapter on its tier, its "
+                  "checksums, and BSR_LOC_HOST");
+  }
   if (c->L == 0) return fail(c, BSR_ERR_STATE, "tier_put before registration");
   if (len != c->chunk_bytes)
     return fail(c, BSR_ERR_INVALID, "tier_put: len %zu != chunk bytes %llu", len,
@@ -1179,6 +1202,14 @@ int bsr_tier_remove_at(bsr_ctx *c, uint32_t tier, uint32_t rank, uint64_t key) {
   if (!c || rank >= c->cfg.n_ranks || tier >= BSR_MAX_TIERS) return BSR_ERR_INVALID;
   std::lock_guard<std::mutex> lk(c->mu);
   c->tier[tier][rank].erase(key);
+  return BSR_OK;
+}
+
+int bsr_tier_set_fetch(bsr_ctx *c, uint32_t tier, bsr_fetch_fn fn, void *user) {
+  if (!c || tier >= BSR_MAX_TIERS) return BSR_ERR_INVALID;
+  std::lock_guard<std::mutex> lk(c->mu);
+  c->fetch_fn[tier] = fn;
+  c->fetch_user[tier] = user;
   return BSR_OK;
 }
 

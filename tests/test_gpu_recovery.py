@@ -158,3 +158,93 @@ def test_lower_tier_is_chosen_for_the_longer_prefix_and_tier_loss_fails_closed()
                 assert bool((c.gpaged[r][l] == synth.CANARY).all())
     finally:
         c.close()
+
+
+def test_file_backed_lower_tier_through_the_fetch_adapter(tmp_path):
+    """The lower tier lives in files (the paper's local-SSD tier): objects are indexed without bytes
+    and a fetch function reads each piece straight into the pinned slot, several reads in flight.
+    The remote tier is down, so the whole request is served from the files, bit-exactly; a read
+    error on one rank fails the request closed."""
+    import ctypes
+    import os
+    import torch
+    from harness import Case, assert_paged_equal, run_oracle
+    from paper_2608_17826_b200 import binding as B
+
+    layout = synth.baseline_layout()                          # 16.4 MB chunks: two fill pieces each
+    Rk, Nk, Wk = 2, 5, 2
+    case = Case(layout, Rk, Nk, seed=79)
+    ora = run_oracle(case, Wk)
+    files = {}
+    for (r, i), p in case.payload.items():
+        path = tmp_path / f"r{r}_k{int(case.keys[i]):016x}.bin"
+        p.tofile(path)
+        files[(r, int(case.keys[i]))] = os.open(path, os.O_RDONLY)
+    calls, fail_on = [], [None]
+
+    def fetch(user, tier, rank, key, offset, length, dst):
+        try:
+            calls.append((tier, rank, key, offset, length))
+            if fail_on[0] == (rank, key):
+                return 5
+            data = os.pread(files[(rank, key)], length, offset)
+            if len(data) != length:
+                return 1
+            ctypes.memmove(dst, data, length)
+            return 0
+        except Exception:                                      # never let an exception read as success
+            return 2
+
+    cb = B.BSR_FETCH_FN(fetch)
+    rc, ctx = B.bsr_ctx_create(Wk, Rk, reg_id=case.reg_id, load_concurrency=4)
+    assert rc == B.BSR_OK
+    dev = torch.device("cuda:0")
+    paged = []
+    try:
+        for r in range(Rk):
+            per = [torch.full((case.pools[g], layout.block_tokens[g], e), synth.CANARY, dtype=torch.uint8, device=dev)
+                   for g, e in layout.tensors]
+            paged.append(per)
+            assert B.bsr_register(ctx, r, [(layout.block_tokens[g], case.pools[g]) for g in range(case.G)],
+                                  [(g, e, per[l].data_ptr()) for l, (g, e) in enumerate(layout.tensors)]) == B.BSR_OK
+        # an object without bytes needs an adapter on its tier
+        assert B.bsr_tier_put_at(ctx, 1, 0, case.keys[0], None, layout.chunk_bytes, case.cks[(0, 0)]) == B.BSR_ERR_INVALID
+        assert B.bsr_tier_set_fetch(ctx, 1, cb) == B.BSR_OK
+        for (r, i) in case.payload:
+            assert B.bsr_tier_put_at(ctx, 1, r, case.keys[i], None, layout.chunk_bytes, case.cks[(r, i)]) == B.BSR_OK
+        assert B.bsr_tier_set_available(ctx, 0, False) == B.BSR_OK           # remote store is down
+        rc, keys, bm, n_hit, tier = B.bsr_probe_request(ctx, 31, case.tok, len(case.tok), case.salt)
+        assert (rc, n_hit, tier) == (B.BSR_OK, Nk, 1) and not calls        # probe fetched nothing
+        flat = [t for tr in case.tables for t in tr]
+        rc, req = B.bsr_req_create(ctx, keys, flat)
+        assert rc == B.BSR_OK and B.bsr_req_bind(ctx, req, 31, tier) == B.BSR_OK
+        assert B.bsr_restore(ctx, req, None) == B.BSR_OK, B.bsr_last_error(ctx)
+        assert B.bsr_commit(ctx, req) == (B.BSR_OK, Nk)
+
+        class _G:                                                           # adapter for assert_paged_equal
+            pass
+        g = _G()
+        g.case, g.paged_numpy = case, (lambda r, l: paged[r][l].cpu().numpy())
+        assert_paged_equal(g, ora["paged"])
+        st = B.bsr_get_stats(ctx)[1]
+        assert st.bytes_restored_by_tier[1] == Rk * Nk * layout.chunk_bytes and st.peak_staging_bytes[0] == Wk * layout.chunk_bytes
+        # every byte of every object was requested exactly once, in pieces of at most 8 MiB
+        got = {}
+        for (t, r, k, off, ln) in calls:
+            assert t == 1 and ln <= 8 << 20
+            got.setdefault((r, k), []).append((off, ln))
+        assert len(got) == Rk * Nk
+        for pieces in got.values():
+            pieces.sort()
+            assert pieces[0][0] == 0 and sum(ln for _, ln in pieces) == layout.chunk_bytes
+            assert all(a[0] + a[1] == b[0] for a, b in zip(pieces, pieces[1:]))
+        # a read error on one rank: zero exposure, marker set
+        fail_on[0] = (1, int(case.keys[3]))
+        assert B.bsr_restore(ctx, req, None) == B.BSR_ERR_TRANSFER
+        assert B.bsr_commit(ctx, req) == (B.BSR_OK, 0)
+        assert B.bsr_request_is_force_local(ctx, 31) == (B.BSR_OK, True)
+        B.bsr_req_release(ctx, req)
+    finally:
+        B.bsr_ctx_destroy(ctx)
+        for fd in files.values():
+            os.close(fd)
