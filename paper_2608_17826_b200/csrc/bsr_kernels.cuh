@@ -232,10 +232,11 @@ bsr_install_vec_kernel(const __grid_constant__ BsrInstallParams p) {
 #define BSR_K_BULK_SMEM (BSR_K_BULK_STAGES * BSR_K_TILE_MAX)
 #define BSR_K_WAIT_NS 2000000000ull  // 2 s: four orders of magnitude above any legitimate wait
 
+// What the producer tells the other warps about the tile it loaded into a stage.
 struct BsrStageMeta {
-  uint64_t dst;    // destination address of the tile (0: no store)
-  uint32_t bytes;  // 0 marks the end of this CTA's work
-  uint32_t word0;
+  uint64_t dst;    // destination address of the tile (unused when the launch only sums)
+  uint32_t bytes;  // tile length
+  uint32_t word0;  // index of the tile's first 32-bit word inside its group segment
   int32_t c;       // chunk descriptor index
   int32_t g;       // group
 };
@@ -289,16 +290,20 @@ __device__ __forceinline__ uint64_t bsr_policy_evict_first() {
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
   return pol;
 }
+// 1-D bulk copy global -> this CTA's shared memory; completion is counted in bytes on `bar`.
+// src, dst and size are multiples of 16 bytes (guaranteed by the tile table).
 __device__ __forceinline__ void bsr_bulk_load(uint32_t smem_dst, const void *gsrc, uint32_t bytes,
-                                                   uint32_t bar, uint64_t pol) {
+                                              uint32_t bar, uint64_t pol) {
   asm volatile(
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, "
       "[%3], %4;" ::"r"(smem_dst),
       "l"(gsrc), "r"(bytes), "r"(bar), "l"(pol)
       : "memory");
 }
+// 1-D bulk copy shared -> global, committed as its own bulk group so that its reads of shared
+// memory can be waited for individually.
 __device__ __forceinline__ void bsr_bulk_store(uint64_t gdst, uint32_t smem_src, uint32_t bytes,
-                                                    uint64_t pol) {
+                                               uint64_t pol) {
   asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;" ::"l"(
                    gdst),
                "r"(smem_src), "r"(bytes), "l"(pol)
