@@ -300,6 +300,9 @@ def run_gpu(args):
 
     # ---- end-to-end arm: tier in host memory, through the pinned W-slot ring ----------------
     h2d_gbs = measure_h2d(torch, dev, chunk)
+    if args.load_concurrency == 0 and world > 1:
+        # several processes share the host cores: split the library's default (half the hardware threads)
+        args.load_concurrency = max(4, min(16, (os.cpu_count() or 8) // 2 // world))
     e2e = Side(B, torch, dev, layout, R, N, W, payload, B.BSR_LOC_HOST,
                load_concurrency=args.load_concurrency, dev_staging_depth=args.depth,
                install_variant=args.variant, direct_install=args.direct)
