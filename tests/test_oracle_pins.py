@@ -216,6 +216,25 @@ def test_peak_is_independent_of_plan_length():
     assert peaks == {8 * reg.slot_bytes}                              # Proposition 1
 
 
+def test_the_papers_scaling_table_rows():
+    """Every row of the paper's W = 32 scaling table: objects = full 256-token chunks of the prefix,
+    external GiB = objects x 16,406,080 B, and the oracle's window loop over that many chunks
+    peaks at 32 slots (500.75 MiB with the 16,408,576-B slot) in K = ceil(objects / 32) windows."""
+    g = read_golden("paper_capacity.txt")
+    per_object = int(g["external_128"]) // 128
+    layout = synth.Layout("narrow", [64], [(0, 16)])               # 4 KiB chunks keep 2,047 of them cheap
+    for key, (objects, gib, mib) in read_golden("paper_scaling_table.txt").items():
+        tokens, objects = int(key[4:]), int(objects)
+        assert tokens // 256 == objects
+        assert round(objects * per_object / 2**30, 3) == float(gib)
+        assert 32 * int(g["law_coefficient"]) == float(mib) * 2**20
+        reg, tok, tiers, keys, tables, paged, _, _ = _build_case(layout, 1, objects, seed=24)
+        req = O.Request(keys[:objects], tables, 1, 1)
+        status, st = O.restore(reg, tiers, req, paged, 32)
+        assert status == O.OK and st.windows == -(-objects // 32)
+        assert st.peak_staging_bytes == [32 * reg.slot_bytes]        # the same for every row
+
+
 def test_w_zero_is_rejected():
     layout = synth.tiny_layout()
     reg, tok, tiers, keys, tables, paged, _, _ = _build_case(layout, 1, 2, seed=23)
