@@ -340,7 +340,8 @@ def run_gpu(args):
     del payload  # 4.2 GB of host memory the oracle leg regenerates for itself
     sample = min(N, 128)  # the whole workload: about 10-20 s of single-thread numpy work
     dt, nbytes = oracle_sample_step(layout, R, sample, W, seed)
-    cpu = {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+    cpu = {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": 1, "host_cores_available": os.cpu_count(),
+           "kind": "oracle",
            "sample": f"first {sample} of {N} chunks x {R} rank slices, one pass ({dt:.1f} s)"}
 
     out = {
