@@ -223,6 +223,15 @@ int bsr_req_release(bsr_ctx *ctx, bsr_req *req);
  * Returns BSR_OK iff every (rank, group, chunk) was verified and installed. */
 int bsr_restore(bsr_ctx *ctx, bsr_req *req, void *cuda_stream);
 
+/* Asynchronous form (Section 3 speaks of "a failed asynchronous restore"): bsr_restore_async starts
+ * the same restore on a thread of the library and returns at once; bsr_restore_wait blocks until it
+ * has finished and stores its status (the value bsr_restore would have returned) in
+ * *restore_status.  One restore per request at a time (STATE otherwise); commit, invalidate and
+ * the observability calls on the request wait for it.  Without an admission budget the restores
+ * of one context still run one after the other. */
+int bsr_restore_async(bsr_ctx *ctx, bsr_req *req, void *cuda_stream);
+int bsr_restore_wait(bsr_ctx *ctx, bsr_req *req, int *restore_status);
+
 /* ---- commit / invalidate (Section 3 "Commit at request semantics", Eq. 6, Proposition 2) -- */
 
 /* exposed_chunks = n_adv_chunks iff a restore of the request completed and all validity bits are

@@ -34,7 +34,7 @@ EXPORTS = [
     "bsr_req_checksums", "bsr_get_stats", "bsr_reset_stats", "bsr_test_inject",
     "bsr_probe_keys_noalloc", "bsr_tier_put_at", "bsr_tier_remove_at", "bsr_tier_set_available",
     "bsr_probe_request", "bsr_req_bind", "bsr_request_done", "bsr_request_is_force_local",
-    "bsr_get_trace", "bsr_tier_set_fetch",
+    "bsr_get_trace", "bsr_tier_set_fetch", "bsr_restore_async", "bsr_restore_wait",
 ]
 # int fn(void *user, uint32 tier, uint32 rank, uint64 key, uint64 offset, uint64 len, void *dst)
 BSR_FETCH_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint64, C.c_uint64,
@@ -120,6 +120,8 @@ def _load() -> C.CDLL:
         "bsr_request_is_force_local": [vp, u64, C.POINTER(i32)],
         "bsr_get_trace": [vp, vp, C.c_size_t, C.POINTER(C.c_size_t)],
         "bsr_tier_set_fetch": [vp, u32, BSR_FETCH_FN, vp],
+        "bsr_restore_async": [vp, vp, vp],
+        "bsr_restore_wait": [vp, vp, C.POINTER(i32)],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -220,6 +222,17 @@ def bsr_req_release(ctx, req) -> int:
 
 def bsr_restore(ctx, req, cuda_stream: int | None = None) -> int:
     return lib.bsr_restore(ctx, req, cuda_stream)
+
+
+def bsr_restore_async(ctx, req, cuda_stream: int | None = None) -> int:
+    return lib.bsr_restore_async(ctx, req, cuda_stream)
+
+
+def bsr_restore_wait(ctx, req):
+    """Returns (rc, status of the restore that was started with bsr_restore_async)."""
+    st = C.c_int(0)
+    rc = lib.bsr_restore_wait(ctx, req, C.byref(st))
+    return rc, st.value
 
 
 def bsr_commit(ctx, req):

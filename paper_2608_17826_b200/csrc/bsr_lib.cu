@@ -122,6 +122,9 @@ struct bsr_req {
   uint64_t request_id = 0;  // engine's request identity (bsr_req_bind); 0 = unbound
   uint32_t tier = 0;        // the one tier this request is served from
   bool bound = false;
+  std::thread async_thread;  // bsr_restore_async: the thread running the restore
+  int async_rc = BSR_OK;
+  bool async_pending = false;
 };
 
 struct bsr_ctx {
@@ -1345,6 +1348,7 @@ int bsr_req_create(bsr_ctx *c, const uint64_t *keys, uint32_t n_adv, const int32
 
 int bsr_req_release(bsr_ctx *c, bsr_req *q) {
   if (!c || !q || q->ctx != c) return BSR_ERR_INVALID;
+  if (q->async_thread.joinable()) q->async_thread.join();  // an asynchronous restore still running
   { std::lock_guard<std::mutex> ql(q->mu); }  // wait for a call in flight on this request
   cudaSetDevice(c->cfg.device);
   cudaFree(q->d_tables);
@@ -1440,8 +1444,26 @@ int bsr_restore(bsr_ctx *c, bsr_req *q, void *cuda_stream) {
   return rc;
 }
 
+int bsr_restore_async(bsr_ctx *c, bsr_req *q, void *cuda_stream) {
+  if (!c || !q || q->ctx != c) return BSR_ERR_INVALID;
+  if (q->async_pending) return fail(c, BSR_ERR_STATE, "restore_async: a restore of this request is pending");
+  q->async_pending = true;
+  q->async_thread = std::thread([c, q, cuda_stream] { q->async_rc = bsr_restore(c, q, cuda_stream); });
+  return BSR_OK;
+}
+
+int bsr_restore_wait(bsr_ctx *c, bsr_req *q, int *restore_status) {
+  if (!c || !q || q->ctx != c) return BSR_ERR_INVALID;
+  if (!q->async_pending) return fail(c, BSR_ERR_STATE, "restore_wait: no restore of this request is pending");
+  if (q->async_thread.joinable()) q->async_thread.join();
+  q->async_pending = false;
+  if (restore_status) *restore_status = q->async_rc;
+  return BSR_OK;
+}
+
 int bsr_commit(bsr_ctx *c, bsr_req *q, uint32_t *exposed) {
   if (!c || !q || q->ctx != c || !exposed) return BSR_ERR_INVALID;
+  if (q->async_thread.joinable()) q->async_thread.join();  // a restore started asynchronously
   std::lock_guard<std::mutex> ql(q->mu);
   bool all = q->restored && !q->failed;
   const uint32_t R = c->cfg.n_ranks;
@@ -1462,6 +1484,7 @@ int bsr_commit(bsr_ctx *c, bsr_req *q, uint32_t *exposed) {
 
 int bsr_invalidate(bsr_ctx *c, bsr_req *q, unsigned flags) {
   if (!c || !q || q->ctx != c) return BSR_ERR_INVALID;
+  if (q->async_thread.joinable()) q->async_thread.join();  // a restore started asynchronously
   std::lock_guard<std::mutex> ql(q->mu);
   invalidate_host(q);
   if ((flags & BSR_SCRUB) && q->n_adv) {
@@ -1493,6 +1516,7 @@ int bsr_invalidate(bsr_ctx *c, bsr_req *q, unsigned flags) {
 
 int bsr_req_bitmap(bsr_ctx *c, bsr_req *q, uint64_t *out, size_t words) {
   if (!c || !q || q->ctx != c || (!out && words)) return BSR_ERR_INVALID;
+  if (q->async_thread.joinable()) q->async_thread.join();  // a restore started asynchronously
   if (words < q->bitmap.size()) return fail(c, BSR_ERR_INVALID, "bitmap buffer too small");
   std::lock_guard<std::mutex> ql(q->mu);
   if (!q->bitmap.empty()) memcpy(out, q->bitmap.data(), q->bitmap.size() * 8);
@@ -1501,6 +1525,7 @@ int bsr_req_bitmap(bsr_ctx *c, bsr_req *q, uint64_t *out, size_t words) {
 
 int bsr_req_checksums(bsr_ctx *c, bsr_req *q, uint64_t *out, size_t count) {
   if (!c || !q || q->ctx != c || (!out && count)) return BSR_ERR_INVALID;
+  if (q->async_thread.joinable()) q->async_thread.join();  // a restore started asynchronously
   const size_t cells = (size_t)c->cfg.n_ranks * c->G * q->n_adv;
   if (count < cells) return fail(c, BSR_ERR_INVALID, "checksum buffer too small");
   std::lock_guard<std::mutex> ql(q->mu);

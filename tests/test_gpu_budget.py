@@ -135,6 +135,28 @@ def test_a_failing_request_fails_alone_under_a_budget():
         c.close()
 
 
+def test_asynchronous_restores_share_the_budget_and_commit_waits_for_them():
+    c = TwoRequests([150, 150], 8, 12)
+    try:
+        B = c.B
+        assert B.bsr_restore_wait(c.ctx, c.greqs[0])[0] == B.BSR_ERR_STATE        # nothing pending
+        for gq in c.greqs:
+            assert B.bsr_restore_async(c.ctx, gq, None) == B.BSR_OK
+        assert B.bsr_restore_async(c.ctx, c.greqs[0], None) == B.BSR_ERR_STATE     # already pending
+        # commit on a request with a restore in flight waits for it instead of exposing zero
+        assert B.bsr_commit(c.ctx, c.greqs[1]) == (B.BSR_OK, 150)
+        statuses = [B.bsr_restore_wait(c.ctx, gq) for gq in c.greqs]
+        assert statuses == [(B.BSR_OK, B.BSR_OK)] * 2
+        opeak = c.compare([s for _, s in statuses])
+        for r in range(R):
+            for l in range(len(c.layout.tensors)):
+                assert np.array_equal(c.gpaged[r][l].cpu().numpy(), c.opaged[r][l])
+        st = B.bsr_get_stats(c.ctx)[1]
+        assert st.peak_staging_bytes[0] == opeak[0] == 12 * c.reg.slot_bytes
+    finally:
+        c.close()
+
+
 def test_four_concurrent_restores_one_failing():
     c = TwoRequests([70, 55, 64, 40], 4, 10, corrupt=(2, 1, 33), load_concurrency=6)
     try:
