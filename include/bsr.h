@@ -251,6 +251,14 @@ int bsr_invalidate(bsr_ctx *ctx, bsr_req *req, unsigned flags);
  * i % 64.  `words` must be at least R*G*ceil(n_adv/64). */
 int bsr_req_bitmap(bsr_ctx *ctx, bsr_req *req, uint64_t *out, size_t words);
 
+/* The destination blocks an engine must treat as erroneous (Section 4 "vLLM failure integration":
+ * a failed retrieve can already have copied a subset of its blocks, so ALL its destination block
+ * ids are recorded).  *count = number of ids of (rank, group): every block of the request's table
+ * once the request has failed or been invalidated, 0 while it is healthy; the first
+ * min(*count, capacity) ids are copied to out. */
+int bsr_req_invalid_blocks(bsr_ctx *ctx, bsr_req *req, uint32_t rank, uint32_t group, int32_t *out,
+                           size_t capacity, size_t *count);
+
 /* Checksums the install kernel computed, out[(r*G + g) * n_adv + i]; 0 where not installed. */
 int bsr_req_checksums(bsr_ctx *ctx, bsr_req *req, uint64_t *out, size_t count);
 

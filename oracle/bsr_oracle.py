@@ -340,6 +340,13 @@ def commit(reg: Registration, req: Request, paged) -> int:
     return 0
 
 
+def invalid_blocks(req: Request, r: int, g: int) -> np.ndarray:
+    """Destination blocks the engine must treat as erroneous (Section 4 "vLLM failure integration"):
+    a failed retrieve may already have copied a subset of its blocks, so ALL block ids of the
+    request's table are reported once it has failed; none while it is healthy."""
+    return req.block_tables[r][g].copy() if req.failed else req.block_tables[r][g][:0].copy()
+
+
 def invalidate(reg: Registration, req: Request, paged, scrub: bool):
     """Whole-prefix invalidation: every bit of every rank and group is cleared, whichever
     component failed.  With scrub, every destination block of the request is zero-filled."""

@@ -35,6 +35,7 @@ EXPORTS = [
     "bsr_probe_keys_noalloc", "bsr_tier_put_at", "bsr_tier_remove_at", "bsr_tier_set_available",
     "bsr_probe_request", "bsr_req_bind", "bsr_request_done", "bsr_request_is_force_local",
     "bsr_get_trace", "bsr_tier_set_fetch", "bsr_restore_async", "bsr_restore_wait",
+    "bsr_req_invalid_blocks",
 ]
 # int fn(void *user, uint32 tier, uint32 rank, uint64 key, uint64 offset, uint64 len, void *dst)
 BSR_FETCH_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint64, C.c_uint64,
@@ -122,6 +123,7 @@ def _load() -> C.CDLL:
         "bsr_tier_set_fetch": [vp, u32, BSR_FETCH_FN, vp],
         "bsr_restore_async": [vp, vp, vp],
         "bsr_restore_wait": [vp, vp, C.POINTER(i32)],
+        "bsr_req_invalid_blocks": [vp, vp, u32, u32, vp, C.c_size_t, C.POINTER(C.c_size_t)],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -249,6 +251,14 @@ def bsr_req_bitmap(ctx, req, n_ranks: int, n_groups: int, n_adv: int):
     out = np.zeros(n_ranks * n_groups * ((n_adv + 63) // 64), dtype=np.uint64)
     rc = lib.bsr_req_bitmap(ctx, req, _ptr(out), out.size)
     return rc, out
+
+
+def bsr_req_invalid_blocks(ctx, req, rank: int, group: int, capacity: int):
+    """Returns (rc, int32 array of the erroneous destination block ids of (rank, group))."""
+    out = np.zeros(max(capacity, 1), dtype=np.int32)
+    n = C.c_size_t(0)
+    rc = lib.bsr_req_invalid_blocks(ctx, req, rank, group, _ptr(out), capacity, C.byref(n))
+    return rc, out[: min(n.value, capacity)]
 
 
 def bsr_req_checksums(ctx, req, n_ranks: int, n_groups: int, n_adv: int):

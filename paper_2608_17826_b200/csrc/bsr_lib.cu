@@ -1514,6 +1514,20 @@ int bsr_invalidate(bsr_ctx *c, bsr_req *q, unsigned flags) {
   return BSR_OK;
 }
 
+int bsr_req_invalid_blocks(bsr_ctx *c, bsr_req *q, uint32_t rank, uint32_t group, int32_t *out,
+                           size_t capacity, size_t *count) {
+  if (!c || !q || q->ctx != c || !count || (!out && capacity)) return BSR_ERR_INVALID;
+  if (rank >= c->cfg.n_ranks || group >= c->G) return fail(c, BSR_ERR_INVALID, "invalid_blocks: rank/group");
+  if (q->async_thread.joinable()) q->async_thread.join();  // a restore started asynchronously
+  std::lock_guard<std::mutex> ql(q->mu);
+  // a failed retrieve may already have copied a subset of its blocks: all of them are erroneous
+  const std::vector<int32_t> &t = q->tables[(size_t)rank * c->G + group];
+  *count = q->failed ? t.size() : 0;
+  const size_t n = *count < capacity ? *count : capacity;
+  if (n) memcpy(out, t.data(), n * sizeof(int32_t));
+  return BSR_OK;
+}
+
 int bsr_req_bitmap(bsr_ctx *c, bsr_req *q, uint64_t *out, size_t words) {
   if (!c || !q || q->ctx != c || (!out && words)) return BSR_ERR_INVALID;
   if (q->async_thread.joinable()) q->async_thread.join();  // a restore started asynchronously

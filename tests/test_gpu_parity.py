@@ -32,6 +32,8 @@ def _check_success(case, W, gpu, ora, n_adv):
             assert st.peak_staging_bytes[r] == 0 and st.bytes_h2d[r] == 0
     assert st.slot_bytes == slot
     assert st.tier_bytes_read_by_probe == 0
+    rc, bad = B.bsr_req_invalid_blocks(gpu.ctx, gpu.req, 0, 0, 8)
+    assert rc == B.BSR_OK and len(bad) == 0           # a healthy request has no erroneous block
 
 
 # ---------------------------------------------------------------- probe
@@ -154,6 +156,10 @@ def _check_failed(case, W, gpu, n_adv, want_rc, scrub_paged):
     B = gpu.B
     assert gpu.commit() == 0
     assert (gpu.bitmap(n_adv) == 0).all()
+    for r in range(case.R):                      # all destination blocks of the request are erroneous
+        for g, t in enumerate(case.tables_prefix(n_adv)[r]):
+            rc, bad = B.bsr_req_invalid_blocks(gpu.ctx, gpu.req, r, g, len(t) + 4)
+            assert rc == B.BSR_OK and np.array_equal(bad, t)
     st = gpu.stats()
     assert 0 < max(st.peak_staging_bytes[: case.R]) <= W * case.reg.slot_bytes
     assert B.bsr_invalidate(gpu.ctx, gpu.req, B.BSR_SCRUB) == B.BSR_OK

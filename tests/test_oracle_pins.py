@@ -377,6 +377,13 @@ def test_failure_cases_are_fail_closed_and_scrub_zeroes_only_request_blocks():
     req = O.Request(keys[:N], tables, R, reg.n_groups)
     status, st = O.restore(reg, tiers, req, paged, W)
     assert status == O.ERR_MISSING and O.commit(reg, req, paged) == 0 and not req.valid.any()
+    # every destination block of the request is erroneous, also those of windows never reached
+    for r in range(R):
+        for g in range(reg.n_groups):
+            assert np.array_equal(O.invalid_blocks(req, r, g), tables[r][g]) and len(tables[r][g]) > 0
+    healthy = O.Request(keys[:3], [[t[: 3 * reg.blocks_per_chunk(g)] for g, t in enumerate(tr)] for tr in tables],
+                        R, reg.n_groups)
+    assert O.restore(reg, tiers, healthy, paged, W)[0] == O.OK and len(O.invalid_blocks(healthy, 0, 0)) == 0
     # the first window (chunks 0..2) was already copied: partial bytes exist, exposure is still zero
     assert np.array_equal(paged[0][0][tables[0][0][0]], payload[(0, 0)][: 16 * 48].reshape(16, 48))
     O.invalidate(reg, req, paged, scrub=True)
