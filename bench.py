@@ -217,7 +217,8 @@ def measure_h2d(torch, dev, piece_bytes, total_bytes=1 << 30, reps=5):
     return best
 
 
-def timed_steps(torch, dist, world, side, tok, n_tok, salt, tok_on_device, steps, warmup, n_chunks):
+def timed_steps(torch, dist, world, side, tok, n_tok, salt, tok_on_device, steps, warmup, n_chunks,
+                coll_dev="cuda"):
     stream = torch.cuda.current_stream()
     for _ in range(warmup):
         side.step(tok, n_tok, salt, tok_on_device, stream.cuda_stream)
@@ -232,14 +233,14 @@ def timed_steps(torch, dist, world, side, tok, n_tok, salt, tok_on_device, steps
         n_hit, exposed = side.step(tok, n_tok, salt, tok_on_device, stream.cuda_stream)
         ok = ok and n_hit == n_chunks and exposed == n_chunks
         if world > 1:  # request-level commit across GPUs: one word, AND over ranks (Eq. 6)
-            ok = ok and multi.commit_across_ranks(exposed, n_chunks, device="cuda") == n_chunks
+            ok = ok and multi.commit_across_ranks(exposed, n_chunks, device=coll_dev) == n_chunks
     e1.record(stream)
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
     ms = e0.elapsed_time(e1)
     if world > 1:
-        ms = multi.max_over_ranks(ms, device="cuda")
+        ms = multi.max_over_ranks(ms, device=coll_dev)
     assert ok, "a step did not expose the full prefix"
     return ms / steps, side.stats()
 
@@ -257,10 +258,18 @@ def run_gpu(args):
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the BSR path has no CPU fallback")
+    if args.dry_run_one_gpu:
+        # plumbing check only: every rank drives GPU 0 and the commit word travels over gloo (NCCL
+        # refuses two ranks on one device).  The ranks' kernels never wait on one another.
+        local = 0
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
+    coll_dev = None if args.dry_run_one_gpu else "cuda"
     if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+        if args.dry_run_one_gpu:
+            dist.init_process_group("gloo")
+        else:
+            dist.init_process_group("nccl", device_id=dev)
 
     layout = {"baseline": synth.baseline_layout, "hetero": synth.hetero_layout,
               "mtp_on": synth.mtp_on_layout}[args.layout]()
@@ -281,7 +290,7 @@ def run_gpu(args):
     sampler = ClockSampler(local)
     sampler.start()
     ms_res, st_res = timed_steps(torch, dist, world, res, d_tok.data_ptr(), len(tok), salt, True,
-                                 args.steps, args.warmup, N)
+                                 args.steps, args.warmup, N, coll_dev)
     launches = int(st_res.kernel_launches)
     k_launches = int(st_res.install_launches)
     k_ms = st_res.install_kernel_ms / max(1, k_launches)
@@ -309,7 +318,7 @@ def run_gpu(args):
     e2e.fill_tier(keys)
     e2e_steps = max(3, min(args.steps, 10))
     ms_e2e, st_e2e = timed_steps(torch, dist, world, e2e, tok, len(tok), salt, False, e2e_steps,
-                                 max(3, min(args.warmup, 3)), N)
+                                 max(3, min(args.warmup, 3)), N, coll_dev)
     peak_staging = [int(st_e2e.peak_staging_bytes[r]) for r in range(R)]
     slot = int(st_e2e.slot_bytes)
     e2e_install_us = 1e3 * st_e2e.install_kernel_ms / max(1, int(st_e2e.install_launches))
@@ -345,6 +354,7 @@ def run_gpu(args):
            "sample": f"first {sample} of {N} chunks x {R} rank slices, one pass ({dt:.1f} s)"}
 
     out = {
+        **({"dry_run_one_gpu": True} if args.dry_run_one_gpu else {}),
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_res, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "u8 payload, u64 checksums/digests", "data": "synthetic",
@@ -441,6 +451,9 @@ def main():
                     help="registration geometry (the contract line is the baseline one)")
     ap.add_argument("--chunks", type=int, default=0, help="prefix length in chunks (default: the workload's 128)")
     ap.add_argument("--direct", action="store_true", help="e2e arm: staging-free install (kernel reads the pinned slots)")
+    ap.add_argument("--dry-run-one-gpu", action="store_true",
+                    help="under torchrun on a single-GPU box: all ranks share GPU 0, gloo for the commit word; "
+                         "checks the multi-process plumbing, the numbers mean nothing")
     ap.add_argument("--sweep", action="store_true", help="e2e GB/s vs W and vs fill concurrency (long prefixes)")
     ap.add_argument("--resident-only", action="store_true", help="small profiling runs: skip e2e and CPU legs")
     args = ap.parse_args()
