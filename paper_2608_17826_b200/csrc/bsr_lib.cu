@@ -36,7 +36,7 @@ namespace {
 using Clock = std::chrono::steady_clock;
 
 constexpr int kInstallThreads = 256;
-constexpr int kInstallUnroll = 4;
+constexpr int kInstallUnroll = 2;  // 32 registers: 8 CTAs of 256 threads resident per SM
 constexpr int kLaunchSlots = 8;  // scratch sets for batched install launches in flight per restore
 constexpr uint32_t kSmCount = 148;
 constexpr uint64_t kPieceBytes = 8ull << 20;  // fill and host-to-device copy granularity
@@ -309,7 +309,7 @@ int launch_install(bsr_ctx *c, const BsrInstallParams &p, cudaStream_t s, StatDe
     bsr_install_bulk_kernel<<<(uint32_t)(total < want ? total : want), BSR_K_BULK_THREADS,
                               BSR_K_BULK_SMEM, s>>>(p);
   } else {
-    const uint64_t want = (uint64_t)kSmCount * 8;
+    const uint64_t want = (uint64_t)kSmCount * 16;  // two full waves of 8 resident CTAs per SM
     bsr_install_vec_kernel<kInstallThreads, kInstallUnroll>
         <<<(uint32_t)(total < want ? total : want), kInstallThreads, 0, s>>>(p);
   }
