@@ -36,7 +36,8 @@ from paper_2608_17826_b200 import multi, synth  # noqa: E402
 WORKLOAD = dict(name="32768-token prefix, 128 chunks x 16,408,576 B, 2 rank slices, W=32, "
                      "baseline 2-group/99-tensor layout, 64-token blocks",
                 n_chunks=128, n_ranks=2, W=32)
-NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = 1.957  # ncu capture of the install kernel, summarised under profiles/
+# dram read + write bytes per payload byte from the ncu captures of the two install kernels (profiles/)
+NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = {"bsr_install_bulk_kernel": 1.957, "bsr_install_vec_kernel": 1.955}
 METRIC, UNIT = "restore GB/s (all rank slices; per-rank = value / rank slices)", "GB/s"
 
 
@@ -287,6 +288,9 @@ def run_gpu(args):
     rc, keys, _, _ = B.bsr_probe(res.ctx, d_tok.data_ptr(), len(tok), salt, True)
     assert rc == B.BSR_OK
     res.fill_tier(keys)
+    rc, in_use = B.bsr_install_kernel_in_use(res.ctx)
+    assert rc == B.BSR_OK
+    kernel_name = "bsr_install_vec_kernel" if in_use == B.BSR_INSTALL_VECTOR else "bsr_install_bulk_kernel"
     sampler = ClockSampler(local)
     sampler.start()
     ms_res, st_res = timed_steps(torch, dist, world, res, d_tok.data_ptr(), len(tok), salt, True,
@@ -300,7 +304,7 @@ def run_gpu(args):
 
     if args.resident_only:  # profiling runs: only the HBM-resident arm, no JSON contract line
         if rank == 0:
-            print(json.dumps({"resident_only": True, "chunks": N, "ms_per_step": ms_res,
+            print(json.dumps({"resident_only": True, "chunks": N, "kernel": kernel_name, "ms_per_step": ms_res,
                               "install_launches": k_launches, "avg_launch_ms": k_ms,
                               "GBps": step_bytes / (ms_res / 1e3) / 1e9}))
         if world > 1:
@@ -342,8 +346,9 @@ def run_gpu(args):
     achieved = 2 * per_launch_payload / (k_ms / 1e3) / 1e9 if k_ms > 0 else None
     # dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of a smaller launch
     # (64 chunk descriptors, a quarter of the timed launch; traffic grows in proportion to the
-    # descriptors processed): 1.0503 GB + 1.0050 GB for 1.0501 GB of payload, i.e. 1.957 B/B.
-    traffic = NCU_DRAM_BYTES_PER_PAYLOAD_BYTE * per_launch_payload
+    # descriptors processed): bulk kernel 1.0503 GB + 1.0050 GB for 1.0501 GB of payload = 1.957 B/B,
+    # vector kernel 1.0502 GB + 1.0026 GB = 1.955 B/B.
+    traffic = NCU_DRAM_BYTES_PER_PAYLOAD_BYTE[kernel_name] * per_launch_payload
 
     # ---- CPU oracle on a bounded sample -----------------------------------------------------
     del payload  # 4.2 GB of host memory the oracle leg regenerates for itself
@@ -378,7 +383,7 @@ def run_gpu(args):
         "staging_residual_bytes": [p - W * slot for p in peak_staging],
         "gpu_launches": launches,
         "roofline": {"bound": "hbm",
-                     "kernel": "bsr_install_vec_kernel" if args.variant == 1 else "bsr_install_bulk_kernel",
+                     "kernel": kernel_name,
                      "achieved": achieved,
                      "peak": hbm_peak, "unit": "GB/s", "frac": (achieved / hbm_peak) if achieved else None,
                      "traffic": traffic, "peak_source": peak_src,

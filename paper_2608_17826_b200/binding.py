@@ -35,7 +35,7 @@ EXPORTS = [
     "bsr_probe_keys_noalloc", "bsr_tier_put_at", "bsr_tier_remove_at", "bsr_tier_set_available",
     "bsr_probe_request", "bsr_req_bind", "bsr_request_done", "bsr_request_is_force_local",
     "bsr_get_trace", "bsr_tier_set_fetch", "bsr_restore_async", "bsr_restore_wait",
-    "bsr_req_invalid_blocks",
+    "bsr_req_invalid_blocks", "bsr_install_kernel_in_use",
 ]
 # int fn(void *user, uint32 tier, uint32 rank, uint64 key, uint64 offset, uint64 len, void *dst)
 BSR_FETCH_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint64, C.c_uint64,
@@ -124,6 +124,7 @@ def _load() -> C.CDLL:
         "bsr_restore_async": [vp, vp, vp],
         "bsr_restore_wait": [vp, vp, C.POINTER(i32)],
         "bsr_req_invalid_blocks": [vp, vp, u32, u32, vp, C.c_size_t, C.POINTER(C.c_size_t)],
+        "bsr_install_kernel_in_use": [vp, C.POINTER(i32)],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -173,6 +174,13 @@ def bsr_register(ctx, rank: int, groups, tensors) -> int:
     g = (bsr_group_desc * len(groups))(*[bsr_group_desc(b, n) for b, n in groups])
     t = (bsr_tensor_desc * len(tensors))(*[bsr_tensor_desc(gg, e, p) for gg, e, p in tensors])
     return lib.bsr_register(ctx, rank, g, len(groups), t, len(tensors))
+
+
+def bsr_install_kernel_in_use(ctx):
+    """Returns (rc, BSR_INSTALL_VECTOR or BSR_INSTALL_BULK)."""
+    v = C.c_int(0)
+    rc = lib.bsr_install_kernel_in_use(ctx, C.byref(v))
+    return rc, v.value
 
 
 def bsr_chunk_bytes(ctx):

@@ -338,6 +338,21 @@ def test_direct_install_from_pinned_slots_matches_oracle(layout_name, R, N, W):
         assert gpu.commit() == 0 and (gpu.bitmap(N) == 0).all()
 
 
+# ---------------------------------------------------------------- kernel choice by registration
+def test_automatic_kernel_choice_follows_the_run_lengths():
+    from paper_2608_17826_b200 import binding as B
+    want = {"baseline": B.BSR_INSTALL_VECTOR, "hetero": B.BSR_INSTALL_BULK, "tiny": B.BSR_INSTALL_BULK}
+    for name, layout in (("baseline", synth.baseline_layout()), ("hetero", synth.hetero_layout()),
+                         ("tiny", synth.tiny_layout())):
+        case = Case(layout, 1, 1, seed=1600)
+        with GpuSide(case, 1) as gpu:
+            assert B.bsr_install_kernel_in_use(gpu.ctx) == (B.BSR_OK, want[name])
+        with GpuSide(case, 1, install_variant=B.BSR_INSTALL_BULK) as gpu:
+            assert B.bsr_install_kernel_in_use(gpu.ctx) == (B.BSR_OK, B.BSR_INSTALL_BULK)
+        with GpuSide(case, 1, install_variant=B.BSR_INSTALL_VECTOR) as gpu:
+            assert B.bsr_install_kernel_in_use(gpu.ctx) == (B.BSR_OK, B.BSR_INSTALL_VECTOR)
+
+
 # ---------------------------------------------------------------- many pipeline shapes
 def test_many_pipeline_shapes_give_the_same_bytes():
     """Seeded sweep over W, fill threads, staging depth, install path and ranks on one small case:
@@ -427,8 +442,9 @@ def test_bounded_wait_inside_the_install_kernel_reports_timeout_and_context_surv
     R, N, W = 2, 6, 4
     case = Case(layout, R, N, seed=1100)
     ora = run_oracle(case, W)
-    with GpuSide(case, W) as gpu:
+    with GpuSide(case, W, install_variant=2) as gpu:          # the waits live in the bulk-copy kernel
         B = gpu.B
+        assert B.bsr_install_kernel_in_use(gpu.ctx) == (B.BSR_OK, B.BSR_INSTALL_BULK)
         rc, keys, bm, n_hit = gpu.probe()
         gpu.request(keys, n_hit)
         assert B.bsr_test_inject(gpu.ctx, B.BSR_INJECT_KERNEL_WAIT, 1, 0, 3, 0) == B.BSR_OK
