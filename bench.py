@@ -312,7 +312,8 @@ def run_gpu(args):
         return 0
 
     # ---- end-to-end arm: tier in host memory, through the pinned W-slot ring ----------------
-    h2d_gbs = measure_h2d(torch, dev, chunk)
+    h2d_gbs = measure_h2d(torch, dev, chunk)                  # the roofline: copies of one chunk each
+    h2d_one_piece = measure_h2d(torch, dev, 1 << 30, reps=3)  # context: a single 1 GiB copy
     if args.load_concurrency == 0 and world > 1:
         # several processes share the host cores: split the library's default (half the hardware threads)
         args.load_concurrency = max(4, min(16, (os.cpu_count() or 8) // 2 // world))
@@ -378,7 +379,8 @@ def run_gpu(args):
                 "d2h_bytes_per_step": N * 8 + R * layout.n_groups * N * 12,
                 "per_rank_GBps": e2e_value / (world * R), "restore_seconds": ms_e2e / 1e3,
                 "install_us_per_chunk_launch": e2e_install_us,
-                "h2d_link_GBps_measured": h2d_gbs, "frac_of_h2d_link": e2e_value / world / h2d_gbs},
+                "h2d_link_GBps_measured": h2d_gbs, "h2d_link_GBps_single_1GiB_copy": h2d_one_piece,
+                "frac_of_h2d_link": e2e_value / world / h2d_gbs},
         "peak_staging_bytes_per_rank": peak_staging, "staging_law_bytes": W * slot,
         "staging_residual_bytes": [p - W * slot for p in peak_staging],
         "gpu_launches": launches,
