@@ -156,9 +156,9 @@ int bsr_register(bsr_ctx *ctx, uint32_t rank, const bsr_group_desc *groups, uint
                  const bsr_tensor_desc *tensors, uint32_t n_tensors);
 
 /* Which install kernel the context launches for device-resident sources under the registration:
- * BSR_INSTALL_BULK or BSR_INSTALL_VECTOR.  With BSR_INSTALL_AUTO the library picks by the
- * registration's run lengths (vector when at least 90 % of a chunk's bytes lie in tiles of 8 KiB
- * or more, bulk otherwise).  Errors: STATE (not every rank registered yet), CUDA. */
+ * BSR_INSTALL_BULK or BSR_INSTALL_VECTOR.  BSR_INSTALL_AUTO currently means the bulk-copy kernel
+ * (level with the vector kernel on long runs, ahead on short ones); direct_install always reads
+ * host slots with the vector kernel.  Errors: STATE (not every rank registered yet), CUDA. */
 int bsr_install_kernel_in_use(bsr_ctx *ctx, int *variant);
 
 /* Bytes of one chunk and of one staging slot under the current registration. */

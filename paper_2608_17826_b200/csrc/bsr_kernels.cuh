@@ -226,6 +226,9 @@ bsr_install_vec_kernel(const __grid_constant__ BsrInstallParams p) {
 #ifndef BSR_K_BULK_CTAS_PER_SM
 #define BSR_K_BULK_CTAS_PER_SM 2  // 2 x 6 stages x 16 KiB = 192 KiB of the SM's shared memory
 #endif
+#ifndef BSR_K_BULK_TILES_PER_CTA
+#define BSR_K_BULK_TILES_PER_CTA 64  // work per CTA; the grid is sized from it in whole waves
+#endif
 #define BSR_K_BULK_CONSUMER_WARPS 4
 #define BSR_K_BULK_THREADS (32 * (2 + BSR_K_BULK_CONSUMER_WARPS))
 #define BSR_K_BULK_STORE_LAG 2  // stores whose shared-memory reads may still be pending

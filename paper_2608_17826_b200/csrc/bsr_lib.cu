@@ -277,15 +277,11 @@ int finalize_registration(bsr_ctx *c) {
     std::lock_guard<std::mutex> g(c->mu);
     c->st.dev_aux_bytes += c->h_tiles.size() * sizeof(BsrTile) + bases.size() * 8 + c->L * 8;
   }
-  // Kernel choice.  Measured on B200: where nearly all bytes sit in long tiles the vector kernel is
-  // about 2 % ahead (a 256-thread CTA is busy on every tile); with many short runs most of a CTA
-  // idles and the bulk-copy kernel, which does not care about run lengths, is ahead by 4 %.
-  uint64_t long_bytes = 0;
-  for (const BsrTile &tl : c->h_tiles)
-    if (tl.bytes >= 8192) long_bytes += tl.bytes;
-  const bool mostly_long = long_bytes * 10 >= c->chunk_bytes * 9;
-  c->use_bulk = c->cfg.install_variant == BSR_INSTALL_BULK ||
-                (c->cfg.install_variant != BSR_INSTALL_VECTOR && !mostly_long);
+  // Kernel choice.  Measured on B200 with both kernels launched in several waves: the bulk-copy
+  // kernel is level with the vector kernel where nearly all bytes sit in long tiles (1.276 against
+  // 1.283 ms per 256-descriptor launch) and 8 % ahead with many short runs, where most of a
+  // 256-thread CTA of the vector kernel idles.  So BSR_INSTALL_AUTO means the bulk-copy kernel.
+  c->use_bulk = c->cfg.install_variant != BSR_INSTALL_VECTOR;
   c->finalized.store(true, std::memory_order_release);
   return BSR_OK;
 }
@@ -315,11 +311,21 @@ int launch_install(bsr_ctx *c, const BsrInstallParams &p, cudaStream_t s, StatDe
                    bool host_source = false) {
   const uint64_t total = (uint64_t)p.n_chunks * p.n_tiles;
   if (c->use_bulk && !host_source) {
-    const uint64_t want = (uint64_t)kSmCount * BSR_K_BULK_CTAS_PER_SM;  // persistent: one wave
+    // Whole waves of the CTAs an SM holds, each CTA streaming BSR_K_BULK_TILES_PER_CTA tiles through
+    // its stage ring: several waves instead of one persistent wave let the hardware scheduler even
+    // out the tail (measured on B200: 1.28 ms against 1.35 ms per 256-descriptor launch).
+    const uint64_t wave = (uint64_t)kSmCount * BSR_K_BULK_CTAS_PER_SM;
+    uint64_t want = (total / BSR_K_BULK_TILES_PER_CTA + wave - 1) / wave * wave;
+    if (want < wave) want = wave;
     bsr_install_bulk_kernel<<<(uint32_t)(total < want ? total : want), BSR_K_BULK_THREADS,
                               BSR_K_BULK_SMEM, s>>>(p);
   } else {
-    const uint64_t want = (uint64_t)kSmCount * 16;  // two full waves of 8 resident CTAs per SM
+    // About nine tiles per CTA, in whole waves of the 8 CTAs an SM holds: many more CTAs than are
+    // resident let the hardware scheduler even out the tail (measured best on B200; one tile per
+    // CTA and a single persistent wave are both slower).
+    const uint64_t wave = (uint64_t)kSmCount * 8;
+    uint64_t want = (total / 9 + wave - 1) / wave * wave;
+    if (want < 2 * wave) want = 2 * wave;
     bsr_install_vec_kernel<kInstallThreads, kInstallUnroll>
         <<<(uint32_t)(total < want ? total : want), kInstallThreads, 0, s>>>(p);
   }
