@@ -53,7 +53,7 @@ struct BsrInstallParams {
   uint32_t blocks_per_chunk[BSR_K_MAX_GROUPS];
   uint64_t *acc;             // scratch [BSR_K_MAX_BATCH][BSR_K_MAX_GROUPS]; zero on entry, zeroed on exit
   unsigned int *ctas_done;   // scratch counter; zero on entry, zeroed on exit
-  unsigned int *err_flag;    // set to nonzero if a bounded wait gave up (bulk variant)
+  unsigned int *err_flag;    // host-mapped word, set to nonzero if a bounded wait gave up (bulk variant)
   uint64_t *ck_out;          // [(r*G + g) * n_adv + i] computed checksum
   uint32_t *verdict;         // same index: 1 verified, 2 mismatch
   uint64_t wait_ns;          // bound of every wait inside the bulk kernel; 0 = BSR_K_WAIT_NS
@@ -283,7 +283,8 @@ __device__ __forceinline__ bool bsr_mbar_wait(uint32_t bar, uint32_t parity, uns
     if (*abort_flag) return false;
     if (bsr_globaltimer() - t0 > wait_ns) {
       *abort_flag = 1;
-      atomicExch(err_flag, 1u);
+      *reinterpret_cast<volatile unsigned int *>(err_flag) = 1u;  // host-mapped word: a plain store
+      __threadfence_system();
       return false;
     }
   }

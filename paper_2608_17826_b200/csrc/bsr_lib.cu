@@ -71,7 +71,9 @@ struct JobRes {
   std::vector<std::pair<cudaEvent_t, cudaEvent_t>> ev_pool;  // launch timing, batched launches
   cudaEvent_t ev_done = nullptr;
   uint64_t *d_acc = nullptr;      // [n_slots][BATCH][GROUPS] checksum accumulators, kept zero
-  unsigned int *d_cnt = nullptr;  // [n_slots] CTA counters, kept zero; [n_slots] = error flag
+  unsigned int *d_cnt = nullptr;  // [n_slots] CTA counters, kept zero
+  unsigned int *h_err = nullptr;  // pinned, device-visible: raised by a kernel wait that gave up
+  unsigned int *d_err = nullptr;  // device alias of h_err
   uint32_t n_slots = 0;
   uint64_t seq = 0;
 };
@@ -302,7 +304,7 @@ void fill_params(bsr_ctx *c, BsrInstallParams &p, JobRes *res, uint32_t slot) {
     p.blocks_per_chunk[g] = BSR_CHUNK_TOKENS / c->groups[g].block_tokens;
   p.acc = res->d_acc + (size_t)slot * BSR_K_MAX_BATCH * BSR_K_MAX_GROUPS;
   p.ctas_done = res->d_cnt + slot;
-  p.err_flag = res->d_cnt + res->n_slots;
+  p.err_flag = res->d_err;
   p.stall_tile = ~0u;
 }
 
@@ -349,17 +351,21 @@ void destroy_res(JobRes *res) {
   if (res->ev_done) cudaEventDestroy(res->ev_done);
   cudaFree(res->d_acc);
   cudaFree(res->d_cnt);
+  if (res->h_err) cudaFreeHost(res->h_err);
   if (res->stream) cudaStreamDestroy(res->stream);
 }
 
 int init_scratch(bsr_ctx *c, JobRes *res, uint32_t n_slots) {
   res->n_slots = n_slots;
   const size_t acc_bytes = (size_t)n_slots * BSR_K_MAX_BATCH * BSR_K_MAX_GROUPS * 8;
-  const size_t cnt_bytes = (n_slots + 1) * sizeof(unsigned int);
+  const size_t cnt_bytes = n_slots * sizeof(unsigned int);
   CU(c, cudaMalloc(&res->d_acc, acc_bytes));
   CU(c, cudaMalloc(&res->d_cnt, cnt_bytes));
   CU(c, cudaMemset(res->d_acc, 0, acc_bytes));
   CU(c, cudaMemset(res->d_cnt, 0, cnt_bytes));
+  CU(c, cudaHostAlloc((void **)&res->h_err, sizeof(unsigned int), cudaHostAllocMapped));
+  CU(c, cudaHostGetDevicePointer((void **)&res->d_err, res->h_err, 0));
+  *res->h_err = 0;
   CU(c, cudaEventCreateWithFlags(&res->ev_done, cudaEventDisableTiming));
   std::lock_guard<std::mutex> g(c->mu);
   c->st.dev_aux_bytes += acc_bytes + cnt_bytes;
@@ -1436,17 +1442,12 @@ int bsr_restore(bsr_ctx *c, bsr_req *q, void *cuda_stream) {
       }
       rc = all_device ? restore_resident(c, q, res, stream, deadline, objs, sd)
                       : restore_ring(c, q, res, stream, deadline, sd);
-      if (c->use_bulk) {
-        // a bounded wait inside the bulk kernel that gave up raised the device-side error flag
-        unsigned int flag = 0;
-        unsigned int *d_flag = res->d_cnt + res->n_slots;
-        if (cudaMemcpy(&flag, d_flag, sizeof flag, cudaMemcpyDeviceToHost) != cudaSuccess) {
-          if (rc == BSR_OK) rc = fail(c, BSR_ERR_CUDA, "reading the kernel error flag failed");
-        } else if (flag) {
-          cudaMemset(d_flag, 0, sizeof flag);
-          if (rc == BSR_OK || rc == BSR_ERR_CHECKSUM)
-            rc = fail(c, BSR_ERR_TIMEOUT, "a bounded wait inside the install kernel gave up");
-        }
+      // a bounded wait inside the bulk kernel that gave up raised the error word (host-mapped; both
+      // restore paths return only after every kernel they launched has been observed complete)
+      if (*reinterpret_cast<volatile unsigned int *>(res->h_err)) {
+        *res->h_err = 0;
+        if (rc == BSR_OK || rc == BSR_ERR_CHECKSUM)
+          rc = fail(c, BSR_ERR_TIMEOUT, "a bounded wait inside the install kernel gave up");
       }
       release_res(c, res);
     } else if (res) {
