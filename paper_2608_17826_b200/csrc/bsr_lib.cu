@@ -167,8 +167,8 @@ struct bsr_ctx {
   uint64_t *h_put_ck = nullptr, *d_put_ck = nullptr;  // pinned [G] sums + verdict dump
   uint32_t *h_put_verdict = nullptr, *d_put_verdict = nullptr;
   unsigned int *d_probe_cnt = nullptr;
-  int32_t *d_tok = nullptr;
-  uint64_t *d_digests = nullptr, *d_keys = nullptr, *h_keys = nullptr;
+  int32_t *h_tok = nullptr, *d_tok = nullptr;  // pinned staging for host token ids + its device alias
+  uint64_t *d_digests = nullptr, *h_keys = nullptr, *d_keys = nullptr;  // keys: pinned + device alias
   size_t probe_cap_chunks = 0;
 
   // slot pool (setup_mu to create, pool_mu to use)
@@ -911,24 +911,27 @@ int probe_impl(bsr_ctx *c, bool request_scoped, uint64_t request_id, const int32
   std::lock_guard<std::mutex> al(c->aux_mu);  // probe scratch is per context
   CU(c, cudaSetDevice(c->cfg.device));
   if (N > c->probe_cap_chunks) {
-    cudaFree(c->d_tok);
+    if (c->h_tok) cudaFreeHost(c->h_tok);
     cudaFree(c->d_digests);
-    cudaFree(c->d_keys);
     if (c->h_keys) cudaFreeHost(c->h_keys);
-    c->d_tok = nullptr;
-    c->d_digests = c->d_keys = c->h_keys = nullptr;
+    c->h_tok = nullptr;
+    c->d_digests = c->h_keys = nullptr;
     c->probe_cap_chunks = 0;
     const size_t cap = round_up(N, 1024);
-    CU(c, cudaMalloc((void **)&c->d_tok, cap * BSR_CHUNK_TOKENS * 4));
+    // Token ids and keys travel through pinned, device-visible host memory: the kernel reads the
+    // ids and writes the keys over the host link itself (4 B per token in, 8 B per chunk out), which
+    // spares two copy submissions and their latency on a call that takes tens of microseconds.
+    CU(c, cudaHostAlloc((void **)&c->h_tok, cap * BSR_CHUNK_TOKENS * 4, cudaHostAllocMapped));
+    CU(c, cudaHostGetDevicePointer((void **)&c->d_tok, c->h_tok, 0));
     CU(c, cudaMalloc((void **)&c->d_digests, cap * 8));
-    CU(c, cudaMalloc((void **)&c->d_keys, cap * 8));
-    CU(c, cudaHostAlloc((void **)&c->h_keys, cap * 8, cudaHostAllocDefault));
+    CU(c, cudaHostAlloc((void **)&c->h_keys, cap * 8, cudaHostAllocMapped));
+    CU(c, cudaHostGetDevicePointer((void **)&c->d_keys, c->h_keys, 0));
     c->probe_cap_chunks = cap;
   }
   const int32_t *d_tok = tok;
   cudaStream_t s = c->own_stream;
   if (!tok_on_device) {
-    CU(c, cudaMemcpyAsync(c->d_tok, tok, N * BSR_CHUNK_TOKENS * 4, cudaMemcpyHostToDevice, s));
+    memcpy(c->h_tok, tok, N * BSR_CHUNK_TOKENS * 4);
     d_tok = c->d_tok;
   }
   // k_-1 = mix64(salt ^ mix64(reg_id)); a scalar, computed once per call
@@ -944,7 +947,6 @@ int probe_impl(bsr_ctx *c, bool request_scoped, uint64_t request_id, const int32
   bsr_probe_kernel<<<grid, BSR_K_PROBE_THREADS, 0, s>>>(d_tok, (uint32_t)N, salt, k_init,
                                                         c->d_digests, c->d_probe_cnt, c->d_keys);
   CU(c, cudaGetLastError());
-  CU(c, cudaMemcpyAsync(c->h_keys, c->d_keys, N * 8, cudaMemcpyDeviceToHost, s));
   CU(c, cudaStreamSynchronize(s));
   // index lookup: keys only; no payload byte is read, nothing is pinned or referenced afterwards
   const size_t words = (N + 63) / 64;
@@ -1055,9 +1057,8 @@ int bsr_ctx_destroy(bsr_ctx *c) {
   if (c->h_put_ck) cudaFreeHost(c->h_put_ck);
   if (c->h_put_verdict) cudaFreeHost(c->h_put_verdict);
   cudaFree(c->d_probe_cnt);
-  cudaFree(c->d_tok);
+  if (c->h_tok) cudaFreeHost(c->h_tok);
   cudaFree(c->d_digests);
-  cudaFree(c->d_keys);
   if (c->h_keys) cudaFreeHost(c->h_keys);
   if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
   if (c->own_stream) cudaStreamDestroy(c->own_stream);
