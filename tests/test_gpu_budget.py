@@ -196,3 +196,46 @@ def test_sequential_restores_with_a_budget_behave_like_the_locked_mode():
         assert st.peak_staging_bytes[0] == 8 * c.reg.slot_bytes        # one at a time: W, not B
     finally:
         c.close()
+
+
+def test_repeated_concurrent_rounds_with_scrubs_in_between_stay_bit_exact():
+    """Six requests restored concurrently, eight rounds over: between rounds some requests are
+    invalidated with a scrub (their blocks zeroed) and all are restored again, alternating the
+    synchronous and the asynchronous call.  Every round ends with every status OK, every commit
+    exposing the whole prefix and the pool whole; the last round is compared byte by byte."""
+    Ns = [33, 20, 47, 8, 26, 40]
+    c = TwoRequests(Ns, 4, 10, load_concurrency=6)
+    try:
+        B = c.B
+        slot = c.reg.slot_bytes
+        for rnd in range(8):
+            if rnd % 2 == 0:
+                statuses = c.run_gpu_concurrently()
+            else:
+                for gq in c.greqs:
+                    assert B.bsr_restore_async(c.ctx, gq, None) == B.BSR_OK
+                statuses = []
+                for gq in c.greqs:
+                    rc, st_ = B.bsr_restore_wait(c.ctx, gq)
+                    assert rc == B.BSR_OK
+                    statuses.append(st_)
+            assert statuses == [B.BSR_OK] * len(Ns), (rnd, statuses)
+            for k, gq in enumerate(c.greqs):
+                assert B.bsr_commit(c.ctx, gq) == (B.BSR_OK, Ns[k])
+            st = B.bsr_get_stats(c.ctx)[1]
+            assert 4 * slot <= max(st.peak_staging_bytes[:R]) <= 10 * slot
+            if rnd < 7:
+                for k in ((rnd, (rnd + 3) % 6)):                     # two requests lose their blocks
+                    assert B.bsr_invalidate(c.ctx, c.greqs[k % 6], B.BSR_SCRUB) == B.BSR_OK
+                    assert B.bsr_commit(c.ctx, c.greqs[k % 6]) == (B.BSR_OK, 0)
+        ostatus, _, _ = O.restore_concurrent(c.reg, c.tiers, c.oreqs, c.opaged, c.W, c.budget)
+        assert ostatus == [O.OK] * len(Ns)
+        for r in range(R):
+            for l in range(len(c.layout.tensors)):
+                assert np.array_equal(c.gpaged[r][l].cpu().numpy(), c.opaged[r][l])
+        # the pool is whole: one restore alone holds exactly W slots again
+        B.bsr_reset_stats(c.ctx)
+        assert B.bsr_restore(c.ctx, c.greqs[2], None) == B.BSR_OK
+        assert B.bsr_get_stats(c.ctx)[1].peak_staging_bytes[0] == 4 * slot
+    finally:
+        c.close()

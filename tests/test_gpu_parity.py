@@ -454,3 +454,41 @@ def test_bounded_wait_inside_the_install_kernel_reports_timeout_and_context_surv
         B.bsr_reset_stats(gpu.ctx)
         assert gpu.restore() == B.BSR_OK                      # one shot: the context is intact
         _check_success(case, W, gpu, ora, N)
+
+
+# ---------------------------------------------------------------- launch-shape corner cases
+@pytest.mark.parametrize("variant,location", [(1, 0), (1, 1), (2, 0), (2, 1)])
+def test_more_tiles_per_chunk_than_ctas_in_the_grid(variant, location):
+    """160 tensors in 16-token blocks = 2,560 runs per chunk, more than the vector kernel's
+    smallest grid: one CTA then handles tiles of the same chunk that belong to different groups
+    and must keep their checksums apart."""
+    layout = synth.Layout("many_runs", [16, 16], [(0, 16)] * 100 + [(1, 32)] * 60)
+    R, N, W = 2, 5, 2
+    case = Case(layout, R, N, seed=1500 + variant)
+    ora = run_oracle(case, W)
+    with GpuSide(case, W, location=location, install_variant=variant) as gpu:
+        rc, keys, bm, n_hit = gpu.probe()
+        gpu.request(keys, n_hit)
+        assert gpu.restore() == gpu.B.BSR_OK, gpu.B.bsr_last_error(gpu.ctx)
+        _check_success(case, W, gpu, ora, N)
+
+
+def test_admission_stops_at_the_first_failure():
+    """After the failing chunk is observed nothing more is admitted: at most the chunks already in
+    the window were fetched, not the remaining hundreds."""
+    layout = synth.tiny_layout()
+    R, N, W, bad = 2, 300, 4, 6
+    case = Case(layout, R, N, seed=1600)
+    with GpuSide(case, W) as gpu:
+        B = gpu.B
+        rc, keys, bm, n_hit = gpu.probe()
+        gpu.request(keys, n_hit)
+        lo, hi = case.reg.segment(0)
+        case.payload[(1, bad)][lo:hi].view("<u4")[5] ^= np.uint32(2)
+        assert gpu.restore() == B.BSR_ERR_CHECKSUM
+        st = gpu.stats()
+        for r in range(R):
+            assert st.bytes_filled[r] <= (bad + 1 + 2 * W) * case.reg.chunk_bytes
+            assert st.bytes_h2d[r] <= (bad + 1 + 2 * W) * case.reg.chunk_bytes
+            assert st.bytes_installed[r] <= (bad + 1 + W) * case.reg.chunk_bytes
+        assert gpu.commit() == 0 and (gpu.bitmap(N) == 0).all()
