@@ -222,7 +222,9 @@ def timed_steps(torch, dist, world, side, tok, n_tok, salt, tok_on_device, steps
                 coll_dev="cuda"):
     stream = torch.cuda.current_stream()
     for _ in range(warmup):
-        side.step(tok, n_tok, salt, tok_on_device, stream.cuda_stream)
+        _, exposed = side.step(tok, n_tok, salt, tok_on_device, stream.cuda_stream)
+        if world > 1:  # the commit exchange is part of a step: warm its communicator up as well
+            multi.commit_across_ranks(exposed, n_chunks, device=coll_dev)
     side.B.bsr_reset_stats(side.ctx)
     if world > 1:
         dist.barrier()
