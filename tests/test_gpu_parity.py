@@ -492,3 +492,34 @@ def test_admission_stops_at_the_first_failure():
             assert st.bytes_h2d[r] <= (bad + 1 + 2 * W) * case.reg.chunk_bytes
             assert st.bytes_installed[r] <= (bad + 1 + W) * case.reg.chunk_bytes
         assert gpu.commit() == 0 and (gpu.bitmap(N) == 0).all()
+
+
+def test_two_contexts_with_different_registrations_restore_at_the_same_time():
+    """Two engines in one process (different geometry, W, kernel variant) restore concurrently on
+    one GPU; neither sees the other: both are bit-exact and each keeps its own staging law."""
+    import threading
+    case_a = Case(synth.tiny_layout(), 2, 60, seed=1800)
+    case_b = Case(synth.hetero_layout(), 1, 7, seed=1801, reg_id=5)
+    ora_a, ora_b = run_oracle(case_a, 4), run_oracle(case_b, 2)
+    with GpuSide(case_a, 4, install_variant=1) as ga, GpuSide(case_b, 2, install_variant=2) as gb:
+        for g in (ga, gb):
+            rc, keys, bm, n_hit = g.probe()
+            assert rc == g.B.BSR_OK and n_hit == g.case.N
+            g.request(keys, n_hit)
+        out = {}
+        gate = threading.Barrier(2)
+
+        def work(name, g):
+            gate.wait()
+            out[name] = [g.restore() for _ in range(3)]
+
+        ts = [threading.Thread(target=work, args=(n, g)) for n, g in (("a", ga), ("b", gb))]
+        [t.start() for t in ts]
+        [t.join() for t in ts]
+        assert out == {"a": [ga.B.BSR_OK] * 3, "b": [ga.B.BSR_OK] * 3}
+        for g, ora, W in ((ga, ora_a, 4), (gb, ora_b, 2)):
+            assert g.commit() == g.case.N
+            assert np.array_equal(g.bitmap(g.case.N), ora["req"].bitmap())
+            assert_paged_equal(g, ora["paged"])
+            st = g.stats()
+            assert st.peak_staging_bytes[0] == W * g.case.reg.slot_bytes == st.ring_bytes_allocated[0]
