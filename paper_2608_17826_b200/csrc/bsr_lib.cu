@@ -124,6 +124,7 @@ struct bsr_req {
   uint64_t request_id = 0;  // engine's request identity (bsr_req_bind); 0 = unbound
   uint32_t tier = 0;        // the one tier this request is served from
   bool bound = false;
+  std::mutex async_mu;       // guards the three fields below
   std::thread async_thread;  // bsr_restore_async: the thread running the restore
   int async_rc = BSR_OK;
   bool async_pending = false;
@@ -261,6 +262,10 @@ int finalize_registration(bsr_ctx *c) {
     }
     off += (uint64_t)BSR_CHUNK_TOKENS * t.bytes_per_token;
   }
+  // the kernels count the tiles of a launch (up to BSR_K_MAX_BATCH chunks) in 32 bits
+  if (c->h_tiles.size() > (1u << 22))
+    return fail(c, BSR_ERR_INVALID, "registration needs %zu tiles per chunk (limit %u)",
+                c->h_tiles.size(), 1u << 22);
   std::vector<uint64_t> bases((size_t)c->cfg.n_ranks * c->L);
   for (uint32_t r = 0; r < c->cfg.n_ranks; ++r)
     for (uint32_t l = 0; l < c->L; ++l) bases[(size_t)r * c->L + l] = c->tensors[l].base[r];
@@ -565,6 +570,12 @@ int ensure_ring(bsr_ctx *c) {
   for (uint32_t k = 0; k < c->cfg.load_concurrency; ++k) c->fillers.emplace_back(filler_main, c);
   c->ring_ready.store(true, std::memory_order_release);
   return BSR_OK;
+}
+
+// Waits for a restore started with bsr_restore_async (its status stays available to bsr_restore_wait).
+void join_async(bsr_req *q) {
+  std::lock_guard<std::mutex> al(q->async_mu);
+  if (q->async_thread.joinable()) q->async_thread.join();
 }
 
 void invalidate_host(bsr_req *q) {
@@ -1380,7 +1391,7 @@ int bsr_req_create(bsr_ctx *c, const uint64_t *keys, uint32_t n_adv, const int32
 
 int bsr_req_release(bsr_ctx *c, bsr_req *q) {
   if (!c || !q || q->ctx != c) return BSR_ERR_INVALID;
-  if (q->async_thread.joinable()) q->async_thread.join();  // an asynchronous restore still running
+  join_async(q);  // an asynchronous restore still running
   { std::lock_guard<std::mutex> ql(q->mu); }  // wait for a call in flight on this request
   cudaSetDevice(c->cfg.device);
   cudaFree(q->d_tables);
@@ -1473,7 +1484,9 @@ int bsr_restore(bsr_ctx *c, bsr_req *q, void *cuda_stream) {
 
 int bsr_restore_async(bsr_ctx *c, bsr_req *q, void *cuda_stream) {
   if (!c || !q || q->ctx != c) return BSR_ERR_INVALID;
+  std::lock_guard<std::mutex> al(q->async_mu);
   if (q->async_pending) return fail(c, BSR_ERR_STATE, "restore_async: a restore of this request is pending");
+  if (q->async_thread.joinable()) q->async_thread.join();
   q->async_pending = true;
   q->async_thread = std::thread([c, q, cuda_stream] { q->async_rc = bsr_restore(c, q, cuda_stream); });
   return BSR_OK;
@@ -1481,6 +1494,7 @@ int bsr_restore_async(bsr_ctx *c, bsr_req *q, void *cuda_stream) {
 
 int bsr_restore_wait(bsr_ctx *c, bsr_req *q, int *restore_status) {
   if (!c || !q || q->ctx != c) return BSR_ERR_INVALID;
+  std::lock_guard<std::mutex> al(q->async_mu);
   if (!q->async_pending) return fail(c, BSR_ERR_STATE, "restore_wait: no restore of this request is pending");
   if (q->async_thread.joinable()) q->async_thread.join();
   q->async_pending = false;
@@ -1490,7 +1504,7 @@ int bsr_restore_wait(bsr_ctx *c, bsr_req *q, int *restore_status) {
 
 int bsr_commit(bsr_ctx *c, bsr_req *q, uint32_t *exposed) {
   if (!c || !q || q->ctx != c || !exposed) return BSR_ERR_INVALID;
-  if (q->async_thread.joinable()) q->async_thread.join();  // a restore started asynchronously
+  join_async(q);  // a restore started asynchronously
   std::lock_guard<std::mutex> ql(q->mu);
   bool all = q->restored && !q->failed;
   const uint32_t R = c->cfg.n_ranks;
@@ -1511,7 +1525,7 @@ int bsr_commit(bsr_ctx *c, bsr_req *q, uint32_t *exposed) {
 
 int bsr_invalidate(bsr_ctx *c, bsr_req *q, unsigned flags) {
   if (!c || !q || q->ctx != c) return BSR_ERR_INVALID;
-  if (q->async_thread.joinable()) q->async_thread.join();  // a restore started asynchronously
+  join_async(q);  // a restore started asynchronously
   std::lock_guard<std::mutex> ql(q->mu);
   invalidate_host(q);
   if ((flags & BSR_SCRUB) && q->n_adv) {
@@ -1545,7 +1559,7 @@ int bsr_req_invalid_blocks(bsr_ctx *c, bsr_req *q, uint32_t rank, uint32_t group
                            size_t capacity, size_t *count) {
   if (!c || !q || q->ctx != c || !count || (!out && capacity)) return BSR_ERR_INVALID;
   if (rank >= c->cfg.n_ranks || group >= c->G) return fail(c, BSR_ERR_INVALID, "invalid_blocks: rank/group");
-  if (q->async_thread.joinable()) q->async_thread.join();  // a restore started asynchronously
+  join_async(q);  // a restore started asynchronously
   std::lock_guard<std::mutex> ql(q->mu);
   // a failed retrieve may already have copied a subset of its blocks: all of them are erroneous
   const std::vector<int32_t> &t = q->tables[(size_t)rank * c->G + group];
@@ -1557,7 +1571,7 @@ int bsr_req_invalid_blocks(bsr_ctx *c, bsr_req *q, uint32_t rank, uint32_t group
 
 int bsr_req_bitmap(bsr_ctx *c, bsr_req *q, uint64_t *out, size_t words) {
   if (!c || !q || q->ctx != c || (!out && words)) return BSR_ERR_INVALID;
-  if (q->async_thread.joinable()) q->async_thread.join();  // a restore started asynchronously
+  join_async(q);  // a restore started asynchronously
   if (words < q->bitmap.size()) return fail(c, BSR_ERR_INVALID, "bitmap buffer too small");
   std::lock_guard<std::mutex> ql(q->mu);
   if (!q->bitmap.empty()) memcpy(out, q->bitmap.data(), q->bitmap.size() * 8);
@@ -1566,7 +1580,7 @@ int bsr_req_bitmap(bsr_ctx *c, bsr_req *q, uint64_t *out, size_t words) {
 
 int bsr_req_checksums(bsr_ctx *c, bsr_req *q, uint64_t *out, size_t count) {
   if (!c || !q || q->ctx != c || (!out && count)) return BSR_ERR_INVALID;
-  if (q->async_thread.joinable()) q->async_thread.join();  // a restore started asynchronously
+  join_async(q);  // a restore started asynchronously
   const size_t cells = (size_t)c->cfg.n_ranks * c->G * q->n_adv;
   if (count < cells) return fail(c, BSR_ERR_INVALID, "checksum buffer too small");
   std::lock_guard<std::mutex> ql(q->mu);
