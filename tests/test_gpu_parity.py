@@ -523,3 +523,25 @@ def test_two_contexts_with_different_registrations_restore_at_the_same_time():
             assert_paged_equal(g, ora["paged"])
             st = g.stats()
             assert st.peak_staging_bytes[0] == W * g.case.reg.slot_bytes == st.ring_bytes_allocated[0]
+
+
+@pytest.mark.parametrize("case_no", range(12))
+def test_random_registrations_match_the_oracle(case_no):
+    """Seeded random geometry: 1-4 groups, block sizes 16...256, 1-5 tensors per group of 16...1,120
+    bytes per token, 1-3 ranks, 1-9 chunks, W 1-5, either kernel, tier in host or device memory."""
+    rng = np.random.Generator(np.random.SFC64(0xB5B5 + case_no))
+    G = int(rng.integers(1, 5))
+    blocks = [int(rng.choice([16, 32, 64, 128, 256])) for _ in range(G)]
+    tensors = [(g, 16 * int(rng.integers(1, 71))) for g in range(G) for _ in range(int(rng.integers(1, 6)))]
+    layout = synth.Layout(f"random{case_no}", blocks, tensors)
+    R, N, W = int(rng.integers(1, 4)), int(rng.integers(1, 10)), int(rng.integers(1, 6))
+    variant, location = 1 + case_no % 2, (case_no // 2) % 2
+    case = Case(layout, R, N, seed=1900 + case_no)
+    ora = run_oracle(case, W)
+    assert ora["status"] == O.OK
+    with GpuSide(case, W, location=location, install_variant=variant) as gpu:
+        rc, keys, bm, n_hit = gpu.probe()
+        assert rc == gpu.B.BSR_OK and n_hit == N and np.array_equal(keys, ora["keys"])
+        gpu.request(keys, n_hit)
+        assert gpu.restore() == gpu.B.BSR_OK, gpu.B.bsr_last_error(gpu.ctx)
+        _check_success(case, W, gpu, ora, N)

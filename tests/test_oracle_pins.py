@@ -7,6 +7,7 @@ import itertools
 
 import numpy as np
 import pytest
+from hypothesis import given, settings, strategies as st
 
 from conftest import read_golden
 from oracle import bsr_oracle as O
@@ -282,6 +283,31 @@ def test_restore_equals_bytewise_definition_on_tiny_input():
             for l, (gg, _) in enumerate(layout.tensors):
                 if gg == g:
                     assert (paged[r][l][spare] == synth.CANARY).all()
+
+
+@settings(max_examples=25, deadline=None, derandomize=True)
+@given(st.data())
+def test_restore_equals_bytewise_definition_on_random_registrations(data):
+    """Random geometry (1-3 groups, block sizes 16...256, 1-3 tensors per group, odd multiples of
+    16 bytes per token), random R, N, W: the window loop lands every byte where the plain
+    definition puts it, peaks at min(N, W) slots and moves exactly N chunks per rank."""
+    G = data.draw(st.integers(1, 3))
+    blocks = [data.draw(st.sampled_from([16, 32, 64, 128, 256])) for _ in range(G)]
+    tensors = [(g, 16 * data.draw(st.integers(1, 3))) for g in range(G)
+               for _ in range(data.draw(st.integers(1, 3)))]
+    layout = synth.Layout("random", blocks, tensors)
+    R, N, W = data.draw(st.integers(1, 2)), data.draw(st.integers(1, 4)), data.draw(st.integers(1, 5))
+    reg, tok, tiers, keys, tables, paged, payload, pools = _build_case(layout, R, N, seed=data.draw(st.integers(1, 99)))
+    req = O.Request(keys[:N], tables, R, reg.n_groups)
+    status, stats = O.restore(reg, tiers, req, paged, W)
+    assert status == O.OK and O.commit(reg, req, paged) == N
+    want = _brute_force_paged(layout, R, N, tables, payload, pools)
+    for r in range(R):
+        for l in range(len(layout.tensors)):
+            assert np.array_equal(paged[r][l], want[r][l])
+        assert stats.peak_staging_bytes[r] == min(N, W) * reg.slot_bytes
+        assert stats.bytes_installed[r] == N * reg.chunk_bytes
+    assert stats.windows == -(-N // W)
 
 
 def test_identity_table_single_tensor_is_a_plain_concatenation():
