@@ -31,3 +31,37 @@ def test_other_ranks_of_the_reference_arm_do_no_work():
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference",
                           "--steps", "1", "--warmup", "3"], capture_output=True, text=True, env=env, timeout=120)
     assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+import pytest
+
+
+@pytest.mark.gpu
+def test_gpu_arm_prints_one_json_line_with_every_contract_key():
+    """The GPU arm on a reduced prefix (32 chunks; the label says so): one JSON line carrying the
+    metric, the end-to-end figure with its copied bytes, launches, clocks, the roofline of the
+    install kernel and the CPU oracle baseline."""
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--chunks", "32", "--steps", "3",
+                          "--warmup", "3"], capture_output=True, text=True, timeout=900)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.strip()]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    for k in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better",
+              "scaling", "vs_baseline", "dtype", "data", "config", "e2e", "gpu_launches", "clocks", "roofline",
+              "cpu_baseline"):
+        assert k in d, k
+    assert d["n_gpus"] == 1 and d["steps"] == 3 and d["warmup"] >= 3 and d["scaling"] == "weak"
+    assert d["value"] > 0 and d["vs_baseline"] is None and d["data"] == "synthetic"
+    assert d["config"]["workload"].startswith("REDUCED to 32 chunks")
+    e = d["e2e"]
+    assert 0 < e["value"] < d["value"] and e["unit"] == d["unit"]
+    assert e["h2d_bytes_per_step"] >= 32 * 2 * 16_408_576 and e["d2h_bytes_per_step"] > 0
+    assert d["gpu_launches"] == 2 * 3                       # one probe and one install launch per step
+    assert set(("sm_mhz", "sm_max_mhz", "reasons")) <= set(d["clocks"])
+    r = d["roofline"]
+    assert r["bound"] == "hbm" and r["unit"] == "GB/s" and r["kernel"] == "bsr_install_bulk_kernel"
+    assert abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9 and 0.5 < r["frac"] < 1.2
+    assert 0.9 < r["traffic"] / (2 * 32 * 2 * 16_408_576) < 1.1     # measured DRAM bytes ~ algorithmic bytes
+    c = d["cpu_baseline"]
+    assert c["kind"] == "oracle" and c["cores"] == 1 and c["value"] > 0 and c["sample"]
