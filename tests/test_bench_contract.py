@@ -1,9 +1,11 @@
-"""The benchmark's reference arm (the CPU oracle) prints one JSON line with the contract's keys.
-Runs on CPU; the GPU arm is exercised on a B200 by the parity tests and by bench.py itself."""
+"""The benchmark prints one JSON line with the contract's keys: the reference arm (the CPU oracle)
+on CPU, the GPU arm on a B200 with a reduced prefix."""
 import json
 import os
 import subprocess
 import sys
+
+import pytest
 
 from conftest import ROOT
 
@@ -31,9 +33,6 @@ def test_other_ranks_of_the_reference_arm_do_no_work():
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference",
                           "--steps", "1", "--warmup", "3"], capture_output=True, text=True, env=env, timeout=120)
     assert out.returncode == 0 and out.stdout.strip() == ""
-
-
-import pytest
 
 
 @pytest.mark.gpu
