@@ -74,7 +74,7 @@ typedef struct bsr_config {
   uint32_t load_concurrency;  /* threads copying tier objects into staging slots (Table 1 "FS
                                  load concurrency": changes throughput, never W or the peak)     */
   uint32_t dev_staging_depth; /* D >= 1 device staging buffers per rank (bounded auxiliary state,
-                                 M_aux of Eq. 4; independent of the prefix length)               */
+                                 M_aux of Eq. 4; independent of the prefix length); 0 = 12       */
   uint32_t timeout_ms;        /* deadline of one bsr_restore call; 0 = 30,000                    */
   uint32_t slot_align;        /* staging slot size = chunk bytes rounded up to this; 0 = 4096    */
   int32_t device;             /* CUDA device ordinal                                             */
@@ -91,7 +91,23 @@ typedef struct bsr_config {
                                  budget (Section 7 "Current concurrency is conservative"): restores
                                  run concurrently and share a pool of B slots per rank; each holds
                                  at most W, together never more than B                            */
+  uint32_t install_batch;     /* chunk descriptors (chunk x rank) one install launch takes on the
+                                 path through the slot pool; 0 = 16.  A launch waits until that many
+                                 chunks have been queued for copying: never more per rank than D or
+                                 W / 4, never fewer than one chunk of every rank, and never while
+                                 nothing else could make progress.  Larger launches run the kernel
+                                 nearer device-copy speed, smaller ones hand slots back sooner.
+                                 Changes throughput only, never W or the peak                      */
+  uint32_t numa_bind;         /* BSR_NUMA_*: placement of the fill threads and the pinned pool      */
 } bsr_config;
+
+/* Host placement.  AUTO: on a host with more than one NUMA node, the fill threads are bound to the
+ * CPUs of the node the context's GPU hangs off (as far as the process' own affinity mask allows)
+ * and the pinned pool is allocated from a thread bound the same way, so that fills and the GPU's
+ * DMA reads stay on one memory controller; a single-node host, or an unknown node, is left alone.
+ * OFF: never bind.  ALWAYS: bind whenever the GPU's node is known.  Only thread affinity and page
+ * placement of this process are touched, never a setting of the GPU or the driver. */
+enum { BSR_NUMA_AUTO = 0, BSR_NUMA_OFF = 1, BSR_NUMA_ALWAYS = 2 };
 
 typedef struct bsr_group_desc {
   uint32_t block_tokens;    /* tokens per paged block; must divide 256                           */
@@ -121,6 +137,9 @@ typedef struct bsr_stats {
   uint64_t bytes_restored_by_tier[BSR_MAX_TIERS]; /* verified and installed, by source tier          */
   double install_kernel_ms;                     /* sum of their device durations (time_kernels)      */
   double last_restore_ms;                       /* host wall time of the last bsr_restore            */
+  uint64_t install_descriptors;                 /* chunk descriptors those install launches carried  */
+  int64_t fill_numa_node;                       /* node the fill threads and the pool are bound to,
+                                                   -1 = not bound (see bsr_config.numa_bind)          */
 } bsr_stats;
 
 /* ---- context ------------------------------------------------------------------------------- */
@@ -135,16 +154,17 @@ int bsr_ctx_create(const bsr_config *cfg, bsr_ctx **out);
  * first (bsr_req_release) and let no call be in flight on it. */
 int bsr_ctx_destroy(bsr_ctx *ctx);
 
-/* Text of the last CUDA or argument error seen by this context (never NULL; valid until the next
- * failing call on the context; read it from the thread that saw the failing call, with no other
- * call running on the context). */
+/* Text of the last CUDA or argument error seen by this context (never NULL).  The returned string
+ * is a copy that belongs to the calling thread and stays valid until that thread calls
+ * bsr_last_error again; calls running on other threads cannot invalidate it.  With several
+ * threads failing on one context the text is that of whichever failed last. */
 const char *bsr_last_error(bsr_ctx *ctx);
 
 /* ---- registration (Section 4: registered tensors in allocator groups, per TP rank) -------- */
 
 /* Registers rank's paged pools.  groups[G] and tensors[L] are host arrays, copied.  Tensors must
  * be listed group-major (all of group 0, then group 1, ...).  All ranks must register the same
- * geometry; only dev_base differs.
+ * geometry; only dev_base differs.  Every group 0..n_groups-1 must own at least one tensor.
  *
  * Chunk byte layout (defined here, the paper only says a chunk "spans the registered per-rank state
  * of its token range"): groups in order; inside a group its tensors in registration order; per
@@ -155,10 +175,12 @@ const char *bsr_last_error(bsr_ctx *ctx);
 int bsr_register(bsr_ctx *ctx, uint32_t rank, const bsr_group_desc *groups, uint32_t n_groups,
                  const bsr_tensor_desc *tensors, uint32_t n_tensors);
 
-/* Which install kernel the context launches for device-resident sources under the registration:
- * BSR_INSTALL_BULK or BSR_INSTALL_VECTOR.  BSR_INSTALL_AUTO currently means the bulk-copy kernel
- * (level with the vector kernel on long runs, ahead on short ones); direct_install always reads
- * host slots with the vector kernel.  Errors: STATE (not every rank registered yet), CUDA. */
+/* Which install kernel the context launches for sources in device memory under the registration:
+ * BSR_INSTALL_BULK or BSR_INSTALL_VECTOR.  BSR_INSTALL_AUTO means the bulk-copy kernel unless more
+ * than half of a chunk's bytes sit in destination runs of at most 1 KiB (which travel as spans of
+ * several runs and are stored with vector stores in either kernel: there the vector kernel is
+ * ahead); direct_install always reads host slots with the vector kernel.
+ * Errors: STATE (not every rank registered yet), CUDA. */
 int bsr_install_kernel_in_use(bsr_ctx *ctx, int *variant);
 
 /* Bytes of one chunk and of one staging slot under the current registration. */
@@ -238,6 +260,19 @@ int bsr_restore(bsr_ctx *ctx, bsr_req *req, void *cuda_stream);
 int bsr_restore_async(bsr_ctx *ctx, bsr_req *req, void *cuda_stream);
 int bsr_restore_wait(bsr_ctx *ctx, bsr_req *req, int *restore_status);
 
+/* Calibration of the host side of a restore (Section 6.5 keeps throughput apart from the capacity
+ * bound: this is the throughput side).  Runs the request's chunks through the same slot pool with
+ * the same fill threads, piece size and admission rule as bsr_restore, but stops early:
+ *   BSR_CAL_FILL      tier -> pinned slot only; a slot is released as soon as it is full
+ *   BSR_CAL_FILL_H2D  ... and slot -> device staging on the copy stream; released when copied
+ * No kernel is launched, so the paged cache, the request's bitmap and its commit state are left as
+ * they are; byte counters are not advanced (the peak meter is: slots were live).  *seconds = host
+ * wall time of the pass.  Comparing request bytes / seconds of the two forms with the link rate
+ * and with a full restore tells which stage bounds a restore on this host.
+ * Errors: INVALID, and whatever a restore can return for a missing key or a failed copy. */
+enum { BSR_CAL_FILL = 1, BSR_CAL_FILL_H2D = 2 };
+int bsr_restore_calibrate(bsr_ctx *ctx, bsr_req *req, int stages, double *seconds);
+
 /* ---- commit / invalidate (Section 3 "Commit at request semantics", Eq. 6, Proposition 2) -- */
 
 /* exposed_chunks = n_adv_chunks iff a restore of the request completed and all validity bits are
@@ -286,6 +321,16 @@ typedef struct bsr_trace_rec {
 /* Copies the timeline of the most recent restore that went through the slot pool (one record per
  * admitted (chunk, rank), in admission order) into out[capacity]; *count = records available. */
 int bsr_get_trace(bsr_ctx *ctx, bsr_trace_rec *out, size_t capacity, size_t *count);
+
+/* Host topology helper behind BSR_NUMA_AUTO (pure host code, no CUDA call): reads
+ * <sysfs_root>/bus/pci/devices/<pci_bus_id>/numa_node into *node (-1 = the platform does not say),
+ * counts the nodes under <sysfs_root>/devices/system/node into *n_nodes (may be NULL) and copies the
+ * node's CPU list ("0-15,32-47", empty when *node < 0) into cpulist[cpulist_cap] (may be NULL).
+ * sysfs_root is "/sys" on a live system; pci_bus_id as cudaDeviceGetPCIBusId prints it (either case).
+ * Errors: INVALID (NULL argument, unparsable file, list longer than the buffer), MISSING (no such
+ * device or node directory). */
+int bsr_numa_of_pci(const char *sysfs_root, const char *pci_bus_id, int *node, char *cpulist,
+                    size_t cpulist_cap, int *n_nodes);
 
 /* ---- host-side failure injection (tests) -------------------------------------------------- */
 

@@ -12,7 +12,9 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libbsr.so")
+# BSR_LIBRARY selects another build of the same source (the tests' small-stage build of the install
+# kernel, see build.py); it must exist, nothing is built or substituted for it.
+LIB_PATH = os.environ.get("BSR_LIBRARY") or os.path.join(_HERE, "libbsr.so")
 
 BSR_OK, BSR_ERR_INVALID, BSR_ERR_MISSING, BSR_ERR_CHECKSUM, BSR_ERR_TIMEOUT = 0, -1, -2, -3, -4
 BSR_ERR_TRANSFER, BSR_ERR_NOMEM, BSR_ERR_ALIGN, BSR_ERR_STATE, BSR_ERR_CUDA = -5, -6, -7, -8, -9
@@ -35,12 +37,14 @@ EXPORTS = [
     "bsr_probe_keys_noalloc", "bsr_tier_put_at", "bsr_tier_remove_at", "bsr_tier_set_available",
     "bsr_probe_request", "bsr_req_bind", "bsr_request_done", "bsr_request_is_force_local",
     "bsr_get_trace", "bsr_tier_set_fetch", "bsr_restore_async", "bsr_restore_wait",
-    "bsr_req_invalid_blocks", "bsr_install_kernel_in_use",
+    "bsr_req_invalid_blocks", "bsr_install_kernel_in_use", "bsr_restore_calibrate", "bsr_numa_of_pci",
 ]
 # int fn(void *user, uint32 tier, uint32 rank, uint64 key, uint64 offset, uint64 len, void *dst)
 BSR_FETCH_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint64, C.c_uint64,
                            C.c_uint64, C.c_void_p)
 BSR_MAX_TIERS = 4
+BSR_CAL_FILL, BSR_CAL_FILL_H2D = 1, 2
+BSR_NUMA_AUTO, BSR_NUMA_OFF, BSR_NUMA_ALWAYS = 0, 1, 2
 BSR_NOALLOC_MAX_CHUNKS = 8192
 
 
@@ -49,7 +53,8 @@ class bsr_config(C.Structure):
                 ("load_concurrency", C.c_uint32), ("dev_staging_depth", C.c_uint32),
                 ("timeout_ms", C.c_uint32), ("slot_align", C.c_uint32), ("device", C.c_int32),
                 ("reg_id", C.c_uint64), ("install_variant", C.c_uint32), ("time_kernels", C.c_uint32),
-                ("direct_install", C.c_uint32), ("budget_slots", C.c_uint32)]
+                ("direct_install", C.c_uint32), ("budget_slots", C.c_uint32),
+                ("install_batch", C.c_uint32), ("numa_bind", C.c_uint32)]
 
 
 class bsr_group_desc(C.Structure):
@@ -70,7 +75,8 @@ class bsr_stats(C.Structure):
                 ("tier_bytes_read_by_probe", C.c_uint64), ("kernel_launches", C.c_uint64),
                 ("h2d_copies", C.c_uint64), ("install_launches", C.c_uint64),
                 ("bytes_restored_by_tier", C.c_uint64 * 4),
-                ("install_kernel_ms", C.c_double), ("last_restore_ms", C.c_double)]
+                ("install_kernel_ms", C.c_double), ("last_restore_ms", C.c_double),
+                ("install_descriptors", C.c_uint64), ("fill_numa_node", C.c_int64)]
 
 
 class bsr_trace_rec(C.Structure):
@@ -80,7 +86,7 @@ class bsr_trace_rec(C.Structure):
 
 
 def _load() -> C.CDLL:
-    if not os.path.exists(LIB_PATH):
+    if not os.path.exists(LIB_PATH) and not os.environ.get("BSR_LIBRARY"):
         try:  # a fresh checkout: compile once with nvcc, in-tree
             from . import build as _build
             _build.build()
@@ -125,6 +131,8 @@ def _load() -> C.CDLL:
         "bsr_restore_wait": [vp, vp, C.POINTER(i32)],
         "bsr_req_invalid_blocks": [vp, vp, u32, u32, vp, C.c_size_t, C.POINTER(C.c_size_t)],
         "bsr_install_kernel_in_use": [vp, C.POINTER(i32)],
+        "bsr_restore_calibrate": [vp, vp, i32, C.POINTER(C.c_double)],
+        "bsr_numa_of_pci": [C.c_char_p, C.c_char_p, C.POINTER(i32), C.c_char_p, C.c_size_t, C.POINTER(i32)],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -152,10 +160,11 @@ def _ptr(a) -> int | None:
 def bsr_ctx_create(W: int, n_ranks: int, *, load_concurrency: int = 0, dev_staging_depth: int = 0,
                    timeout_ms: int = 0, slot_align: int = 0, device: int = 0, reg_id: int = 1,
                    install_variant: int = BSR_INSTALL_AUTO, time_kernels: bool = False,
-                   direct_install: bool = False, budget_slots: int = 0):
+                   direct_install: bool = False, budget_slots: int = 0, install_batch: int = 0,
+                   numa_bind: int = BSR_NUMA_AUTO):
     cfg = bsr_config(W, n_ranks, BSR_CHUNK_TOKENS, load_concurrency, dev_staging_depth, timeout_ms,
                      slot_align, device, reg_id, install_variant, int(time_kernels),
-                     int(direct_install), budget_slots)
+                     int(direct_install), budget_slots, install_batch, numa_bind)
     ctx = C.c_void_p()
     rc = lib.bsr_ctx_create(C.byref(cfg), C.byref(ctx))
     return rc, (ctx if rc == BSR_OK else None)
@@ -232,6 +241,22 @@ def bsr_req_release(ctx, req) -> int:
 
 def bsr_restore(ctx, req, cuda_stream: int | None = None) -> int:
     return lib.bsr_restore(ctx, req, cuda_stream)
+
+
+def bsr_restore_calibrate(ctx, req, stages: int):
+    """Returns (rc, seconds) of a fill-only or fill + copy pass over the request's chunks."""
+    sec = C.c_double(0.0)
+    rc = lib.bsr_restore_calibrate(ctx, req, stages, C.byref(sec))
+    return rc, sec.value
+
+
+def bsr_numa_of_pci(sysfs_root: str, pci_bus_id: str):
+    """Returns (rc, node, cpulist, n_nodes) read from a sysfs tree (host only, no CUDA call)."""
+    node, n_nodes = C.c_int(-1), C.c_int(0)
+    buf = C.create_string_buffer(1024)
+    rc = lib.bsr_numa_of_pci(sysfs_root.encode(), pci_bus_id.encode(), C.byref(node), buf, len(buf),
+                             C.byref(n_nodes))
+    return rc, node.value, buf.value.decode(), n_nodes.value
 
 
 def bsr_restore_async(ctx, req, cuda_stream: int | None = None) -> int:

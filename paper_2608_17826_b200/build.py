@@ -29,17 +29,39 @@ def up_to_date() -> bool:
     return os.path.exists(LIB) and all(os.path.getmtime(LIB) >= os.path.getmtime(d) for d in DEPS)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and up_to_date():
-        return LIB
-    cmd = [nvcc(), *NVCC_FLAGS, "-o", LIB, SRC]
+def _compile(out: str, defines: list[str], verbose: bool) -> str:
+    cmd = [nvcc(), *NVCC_FLAGS, *defines, "-o", out, SRC]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
         raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
     if verbose:
         sys.stderr.write(res.stdout + res.stderr)
-    return LIB
+    return out
+
+
+def build(force: bool = False, verbose: bool = False) -> str:
+    if not force and up_to_date():
+        return LIB
+    return _compile(LIB, [], verbose)
+
+
+# A second build of the same source for the tests: the bulk install kernel with a ring of only
+# three 1 KiB stages, one lagging store and at most 32 CTAs per launch, so that every shared-memory
+# stage is recycled hundreds of times per CTA (the product build recycles a 16 KiB stage about ten
+# times).  An ordering slip between a stage's store, its checksum and its next load has hundreds of
+# chances per CTA to show as a wrong byte or sum here.
+STRESS_LIB = os.path.join(HERE, "libbsr_stress.so")
+STRESS_DEFINES = ["-DBSR_K_BULK_STAGES=3", "-DBSR_K_BULK_STORE_LAG=1", "-DBSR_K_TILE_MAX=1024u",
+                  "-DBSR_K_BULK_TILES_PER_CTA=512", "-DBSR_K_BULK_MAX_GRID=32"]
+
+
+def build_stress(force: bool = False, verbose: bool = False) -> str:
+    fresh = os.path.exists(STRESS_LIB) and all(os.path.getmtime(STRESS_LIB) >= os.path.getmtime(d) for d in DEPS)
+    if not force and fresh:
+        return STRESS_LIB
+    return _compile(STRESS_LIB, STRESS_DEFINES, verbose)
 
 
 if __name__ == "__main__":
     print(build(force=True, verbose=True))
+    print(build_stress(force=True))

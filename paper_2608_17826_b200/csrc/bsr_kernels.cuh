@@ -12,26 +12,56 @@
 #ifndef BSR_K_TILE_MAX
 #define BSR_K_TILE_MAX 16384u     // largest tile in bytes (one bulk-copy stage)
 #endif
+#ifndef BSR_K_SPAN_RUN_MAX
+#define BSR_K_SPAN_RUN_MAX 1024u  // destination runs up to this length travel as spans of several runs
+#endif
 #define BSR_K_PHI 0x9E3779B97F4A7C15ull
 
 // ---------------------------------------------------------------------------------------------
 // shared structs (host fills, device reads)
 // ---------------------------------------------------------------------------------------------
 
-// One piece of one destination run.  A chunk's tile table is the same for every chunk and rank of
-// a registration: only the source base, the block-table row and the tensor base pointers change.
+// One contiguous span of a chunk, at most BSR_K_TILE_MAX bytes, that is moved as a unit.  Either a
+// piece of ONE destination run (n_runs == 1: long runs are cut into pieces), or n_runs > 1 WHOLE
+// runs that lie back to back in the chunk: the blocks of one tensor and, where consecutive tensors
+// of a group have the same bytes per token, of the tensors that follow it.  Run j of such a span
+// belongs to tensor `tensor + (blk + j) / blocks_per_chunk` and logical block
+// `(blk + j) % blocks_per_chunk`.  Short runs (256 bytes for 16 B/token in 16-token blocks) thus
+// still travel in spans of up to 16 KiB; only their stores are scattered.
+// A chunk's tile table is the same for every chunk and rank of a registration: only the source
+// base, the block-table row and the tensor base pointers change.
 struct __align__(16) BsrTile {
   uint32_t src_off;    // byte offset inside the chunk (multiple of 16)
-  uint32_t bytes;      // tile length (multiple of 16, <= BSR_K_TILE_MAX)
-  uint32_t dst_off;    // byte offset inside the destination block run
-  uint32_t word0;      // index of the tile's first 32-bit word inside its group segment
-  uint32_t run_bytes;  // block_tokens * bytes_per_token of the tensor
-  uint16_t tensor;     // registration index l
+  uint32_t bytes;      // span length (multiple of 16, <= BSR_K_TILE_MAX)
+  uint32_t dst_off;    // byte offset inside the destination block run (0 when n_runs > 1)
+  uint32_t word0;      // index of the span's first 32-bit word inside its group segment
+  uint32_t run_bytes;  // block_tokens * bytes_per_token of the tensor(s)
+  uint16_t tensor;     // registration index l of the first run
   uint8_t group;       // allocator group g
-  uint8_t blk;         // logical block of the chunk, 0 .. 256/block_tokens - 1
-  uint32_t pad[2];
+  uint8_t blk;         // logical block of the first run, 0 .. 256/block_tokens - 1
+  uint32_t n_runs;     // runs in the span
+  uint32_t run_inv;    // ceil(2^32 / run_bytes): byte offset -> run index without a division
 };
 static_assert(sizeof(BsrTile) == 32, "tile is two 16-byte loads");
+
+// Where vector v (16 bytes) of a span of several whole runs goes.
+struct BsrRunMap {
+  const int32_t *tab;     // block-table row of the chunk: table(rank, group) + chunk * blocks_per_chunk
+  const uint64_t *bases;  // tensor base addresses of the rank: tensor_base + rank * n_tensors
+  uint32_t run_bytes, run_inv;
+  uint32_t l0, b0;        // tensor and logical block of the span's first run
+  uint32_t nb_shift;      // log2(blocks per chunk of the group)
+};
+__device__ __forceinline__ uint4 *bsr_run_dst(const BsrRunMap &m, uint32_t v) {
+  const uint32_t off = v << 4;
+  const uint32_t j = __umulhi(off, m.run_inv);  // exact for off < 2^16 and run_bytes >= 256
+  const uint32_t within = off - j * m.run_bytes;
+  const uint32_t vb = m.b0 + j;
+  const uint32_t l = m.l0 + (vb >> m.nb_shift), blk = vb & ((1u << m.nb_shift) - 1u);
+  const uint64_t base = __ldg(m.bases + l);
+  const int32_t phys = __ldg(m.tab + blk);
+  return reinterpret_cast<uint4 *>(base + (uint64_t)phys * m.run_bytes + within);
+}
 
 struct BsrChunkDesc {
   const uint8_t *src;  // device address of the staged chunk
@@ -155,8 +185,10 @@ __device__ __forceinline__ void bsr_install_finish(const BsrInstallParams &p) {
 // ---------------------------------------------------------------------------------------------
 // install, vector variant: 16-byte streaming loads and stores, UNROLL vectors in flight per thread
 // ---------------------------------------------------------------------------------------------
-template <int THREADS, int UNROLL>
-__global__ void __launch_bounds__(THREADS)
+// SPANS: the registration has spans of several runs (their per-vector destination lookup costs
+// registers that a registration of long runs alone should not pay for).
+template <int THREADS, int UNROLL, bool SPANS>
+__global__ void __launch_bounds__(THREADS, 2048 / THREADS)  // full occupancy: 32 registers at 256 threads
 bsr_install_vec_kernel(const __grid_constant__ BsrInstallParams p) {
   __shared__ uint64_t red[THREADS / 32];
   const uint32_t total = p.n_chunks * p.n_tiles;
@@ -168,7 +200,7 @@ bsr_install_vec_kernel(const __grid_constant__ BsrInstallParams p) {
     const uint4 t0 = __ldg(tp), t1 = __ldg(tp + 1);
     const uint32_t src_off = t0.x, bytes = t0.y, dst_off = t0.z, word0 = t0.w;
     const uint32_t run_bytes = t1.x, tensor = t1.y & 0xffffu, g = (t1.y >> 16) & 0xffu,
-                   blk = t1.y >> 24;
+                   blk = t1.y >> 24, n_runs = t1.z;
     if ((int)c != cur_c || (int)g != cur_g) {  // block-uniform
       if (cur_c >= 0) bsr_block_flush<THREADS>(sum, p.acc + cur_c * BSR_K_MAX_GROUPS + cur_g, red);
       sum = 0;
@@ -178,11 +210,23 @@ bsr_install_vec_kernel(const __grid_constant__ BsrInstallParams p) {
     const BsrChunkDesc &cd = *bsr_desc(p, c);
     const uint4 *src = reinterpret_cast<const uint4 *>(cd.src + src_off);
     uint4 *dst = nullptr;
+    BsrRunMap rm;
+    const bool several = SPANS && p.scatter && n_runs > 1;  // whole runs, each with its own destination
     if (p.scatter) {
-      const int32_t *table = p.tables[cd.rank * p.n_groups + g];
-      const int32_t phys = __ldg(table + (size_t)cd.chunk * p.blocks_per_chunk[g] + blk);
-      const uint64_t base = __ldg(p.tensor_base + (size_t)cd.rank * p.n_tensors + tensor);
-      dst = reinterpret_cast<uint4 *>(base + (uint64_t)phys * run_bytes + dst_off);
+      const uint32_t nb = p.blocks_per_chunk[g];
+      const int32_t *row = p.tables[cd.rank * p.n_groups + g] + (size_t)cd.chunk * nb;
+      const uint64_t *bases = p.tensor_base + (size_t)cd.rank * p.n_tensors;
+      if (several) {
+        rm.tab = row;
+        rm.bases = bases;
+        rm.run_bytes = run_bytes;
+        rm.run_inv = t1.w;
+        rm.l0 = tensor;
+        rm.b0 = blk;
+        rm.nb_shift = 31u - __clz(nb);
+      } else {
+        dst = reinterpret_cast<uint4 *>(__ldg(bases + tensor) + (uint64_t)__ldg(row + blk) * run_bytes + dst_off);
+      }
     }
     const uint32_t nvec = bytes >> 4;
     for (uint32_t v0 = threadIdx.x; v0 < nvec; v0 += THREADS * UNROLL) {
@@ -196,7 +240,10 @@ bsr_install_vec_kernel(const __grid_constant__ BsrInstallParams p) {
       for (int u = 0; u < UNROLL; ++u) {
         const uint32_t v = v0 + u * THREADS;
         if (v < nvec) {
-          if (dst) bsr_st_stream(dst + v, r[u]);
+          if (several)
+            bsr_st_stream(bsr_run_dst(rm, v), r[u]);
+          else if (dst)
+            bsr_st_stream(dst + v, r[u]);
           sum += bsr_ck_vec(r[u], word0 + 4u * v);
         }
       }
@@ -212,10 +259,13 @@ bsr_install_vec_kernel(const __grid_constant__ BsrInstallParams p) {
 // addresses and issues the loads, a store warp issues the stores, and four warps sum the tile from
 // shared memory while its store is in flight.
 //
-//   warp 0, producer:  wait empty[s] -> expect_tx(full[s], bytes) -> bulk load tile into stage s
-//   warp 1, storer:    wait full[s]  -> bulk store stage s -> dst; once the store issued two tiles
+//   warp 0, producer:  wait empty[s] -> expect_tx(full[s], bytes) -> bulk load span into stage s
+//   warp 1, storer:    wait full[s]  -> bulk store stage s -> dst; once the store issued two spans
 //                      earlier has finished reading its stage -> arrive empty[that stage]
 //   warps 2.., sums:   wait full[s]  -> checksum from shared memory -> arrive empty[s]
+// A span of several short runs has no single destination: the sum warps, which hold every vector
+// of the stage in registers anyway, store it to the run it belongs to (16-byte streaming stores,
+// a half-warp per 256 bytes), and the storer only hands the stage back.
 //
 // Every wait is bounded by a wall-clock deadline; a wait that gives up raises *err_flag, the CTA
 // stops issuing work, drains what it has in flight and leaves through the common exit.
@@ -231,18 +281,38 @@ bsr_install_vec_kernel(const __grid_constant__ BsrInstallParams p) {
 #endif
 #define BSR_K_BULK_CONSUMER_WARPS 4
 #define BSR_K_BULK_THREADS (32 * (2 + BSR_K_BULK_CONSUMER_WARPS))
+#ifndef BSR_K_BULK_STORE_LAG
 #define BSR_K_BULK_STORE_LAG 2  // stores whose shared-memory reads may still be pending
+#endif
 #define BSR_K_BULK_SMEM (BSR_K_BULK_STAGES * BSR_K_TILE_MAX)
+// A stage is handed back to the producer only LAG stores after its own store was issued: with as
+// many lagging stores as stages the producer would wait for a stage nobody is about to release.
+static_assert(BSR_K_BULK_STAGES > BSR_K_BULK_STORE_LAG, "the stage ring must be deeper than the store lag");
+static_assert(BSR_K_BULK_STORE_LAG >= 0 && BSR_K_BULK_STORE_LAG <= 5, "the storer packs LAG + 1 stage numbers into 32 bits");
+static_assert(BSR_K_TILE_MAX % 128u == 0 && BSR_K_TILE_MAX >= 256u, "tiles are cut on 128-byte boundaries");
 #define BSR_K_WAIT_NS 2000000000ull  // 2 s: four orders of magnitude above any legitimate wait
 
-// What the producer tells the other warps about the tile it loaded into a stage.
-struct BsrStageMeta {
-  uint64_t dst;    // destination address of the tile (unused when the launch only sums)
-  uint32_t bytes;  // tile length
-  uint32_t word0;  // index of the tile's first 32-bit word inside its group segment
-  int32_t c;       // chunk descriptor index
-  int32_t g;       // group
+// What the producer tells the other warps about the span it loads into a stage.  One entry per
+// span in flight, in a ring indexed by the CTA's span counter: entries are written 32 at a time by
+// the lanes that resolve them, and a slot is rewritten only 64 spans later, long after the other
+// warps (at most a stage ring behind the producer) are done with it.
+#define BSR_K_META_RING 64
+struct __align__(16) BsrStageMeta {
+  uint64_t src;           // source address of the span
+  uint64_t dst;           // one run: destination address of the piece (0 when the launch only sums)
+  const int32_t *tab;     // several runs: see BsrRunMap
+  const uint64_t *bases;
+  uint32_t bytes;         // span length
+  uint32_t word0;         // index of the span's first 32-bit word inside its group segment
+  uint32_t run_bytes, run_inv;
+  uint16_t l0, b0;
+  uint16_t nb_shift;
+  uint16_t several;       // nonzero: whole runs with their own destinations, stored by the sum warps
+  uint32_t cg;            // chunk descriptor index << 8 | group
+  uint32_t pad;
 };
+static_assert(sizeof(BsrStageMeta) == 64, "four 16-byte words per entry");
+static_assert(BSR_K_BULK_STAGES <= 32, "the meta ring assumes the other warps trail the producer by < 32 spans");
 
 __device__ __forceinline__ uint32_t bsr_smem_u32(const void *p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -320,7 +390,7 @@ bsr_install_bulk_kernel(const __grid_constant__ BsrInstallParams p) {
   extern __shared__ __align__(128) uint8_t stage_mem[];
   __shared__ __align__(8) uint64_t full_bar[BSR_K_BULK_STAGES];
   __shared__ __align__(8) uint64_t empty_bar[BSR_K_BULK_STAGES];
-  __shared__ BsrStageMeta meta[BSR_K_BULK_STAGES];
+  __shared__ BsrStageMeta meta[BSR_K_META_RING];
   __shared__ int last_round[BSR_K_BULK_STAGES];  // last load round issued into each stage, -1 = none
   __shared__ int abort_flag;
 
@@ -345,86 +415,107 @@ bsr_install_bulk_kernel(const __grid_constant__ BsrInstallParams p) {
 
   if (warp == 0) {
     // ---------------- producer ----------------
-    // The address of a tile needs a chain of dependent loads (tile entry -> block table -> tensor
-    // base).  The 32 lanes resolve 32 consecutive tiles of this CTA at once; lane 0 then issues them
-    // in order, taking each tile's values from the lane that resolved it.
+    // The address of a span needs a chain of dependent loads (tile entry -> block table -> tensor
+    // base).  The 32 lanes resolve 32 consecutive spans of this CTA at once, each into its own
+    // entry of the meta ring; lane 0 then issues the loads in order.
     for (uint32_t base = 0; base < my_tiles; base += 32) {
       const uint32_t n_mine = base + lane;
-      uint64_t src = 0, dst = 0;
-      uint32_t bytes = 0, word0 = 0, cg = 0;
       if (n_mine < my_tiles) {
         const uint32_t w = blockIdx.x + n_mine * gridDim.x;
         const uint32_t c = w / p.n_tiles, t = w - c * p.n_tiles;
         const uint4 *tp = reinterpret_cast<const uint4 *>(p.tiles + t);
         const uint4 t0 = __ldg(tp), t1 = __ldg(tp + 1);
-        const uint32_t g = (t1.y >> 16) & 0xffu;
+        const uint32_t g = (t1.y >> 16) & 0xffu, tensor = t1.y & 0xffffu, blk = t1.y >> 24;
         const BsrChunkDesc &cd = *bsr_desc(p, c);
+        BsrStageMeta m;
+        m.src = reinterpret_cast<uint64_t>(cd.src) + t0.x;
+        m.dst = 0;
+        m.tab = nullptr;
+        m.bases = nullptr;
+        m.bytes = t0.y;
+        m.word0 = t0.w;
+        m.run_bytes = t1.x;
+        m.run_inv = t1.w;
+        m.l0 = (uint16_t)tensor;
+        m.b0 = (uint16_t)blk;
+        m.nb_shift = 0;
+        m.several = 0;
+        m.cg = (c << 8) | g;
+        m.pad = 0;
         if (p.scatter) {
-          const int32_t *table = p.tables[cd.rank * p.n_groups + g];
-          const int32_t phys = __ldg(table + (size_t)cd.chunk * p.blocks_per_chunk[g] + (t1.y >> 24));
-          dst = __ldg(p.tensor_base + (size_t)cd.rank * p.n_tensors + (t1.y & 0xffffu)) +
-                (uint64_t)phys * t1.x + t0.z;
+          const uint32_t nb = p.blocks_per_chunk[g];
+          const int32_t *row = p.tables[cd.rank * p.n_groups + g] + (size_t)cd.chunk * nb;
+          const uint64_t *bases = p.tensor_base + (size_t)cd.rank * p.n_tensors;
+          if (t1.z > 1) {
+            m.tab = row;
+            m.bases = bases;
+            m.nb_shift = (uint16_t)(31u - __clz(nb));
+            m.several = 1;
+          } else {
+            m.dst = __ldg(bases + tensor) + (uint64_t)__ldg(row + blk) * t1.x + t0.z;
+          }
         }
-        src = reinterpret_cast<uint64_t>(cd.src) + t0.x;
-        bytes = t0.y;
-        word0 = t0.w;
-        cg = (c << 8) | g;
+        meta[n_mine % BSR_K_META_RING] = m;
       }
+      __syncwarp();  // lane 0 publishes the other lanes' entries with its barrier arrivals below
       const uint32_t cnt = min(32u, my_tiles - base);
       int ok = 1;
-      for (uint32_t j = 0; j < cnt && ok; ++j) {
-        const uint64_t src_j = __shfl_sync(0xffffffffu, src, j);
-        const uint64_t dst_j = __shfl_sync(0xffffffffu, dst, j);
-        const uint32_t bytes_j = __shfl_sync(0xffffffffu, bytes, j);
-        const uint32_t word0_j = __shfl_sync(0xffffffffu, word0, j);
-        const uint32_t cg_j = __shfl_sync(0xffffffffu, cg, j);
-        if (lane == 0) {
+      if (lane == 0) {
+        for (uint32_t j = 0; j < cnt; ++j) {
           const uint32_t n = base + j;
           const uint32_t s = n % BSR_K_BULK_STAGES, round = n / BSR_K_BULK_STAGES;
           if (round > 0 &&
               !bsr_mbar_wait(bsr_smem_u32(&empty_bar[s]), (round - 1) & 1u, p.err_flag, &abort_flag, wait_ns)) {
             ok = 0;
-          } else if (blockIdx.x + n * gridDim.x == p.stall_tile) {
-            // test hook: this tile's load is never issued, so the waits on its stage run out
-          } else {
-            meta[s].dst = dst_j;
-            meta[s].bytes = bytes_j;
-            meta[s].word0 = word0_j;
-            meta[s].c = (int32_t)(cg_j >> 8);
-            meta[s].g = (int32_t)(cg_j & 0xffu);
-            const uint32_t bar = bsr_smem_u32(&full_bar[s]);
-            bsr_mbar_expect_tx(bar, bytes_j);  // release: the meta writes above are visible to waiters
-            bsr_bulk_load(bsr_smem_u32(stage_mem + (size_t)s * BSR_K_TILE_MAX),
-                          reinterpret_cast<const void *>(src_j), bytes_j, bar, pol);
-            last_round[s] = (int)round;
+            break;
           }
+          if (blockIdx.x + n * gridDim.x == p.stall_tile) continue;  // test hook: never loaded, its waits run out
+          const BsrStageMeta &m = meta[n % BSR_K_META_RING];
+          const uint32_t bar = bsr_smem_u32(&full_bar[s]);
+          bsr_mbar_expect_tx(bar, m.bytes);  // release: the meta entry is visible to whoever sees the stage full
+          bsr_bulk_load(bsr_smem_u32(stage_mem + (size_t)s * BSR_K_TILE_MAX),
+                        reinterpret_cast<const void *>(m.src), m.bytes, bar, pol);
+          last_round[s] = (int)round;
         }
-        ok = __shfl_sync(0xffffffffu, ok, 0);
       }
+      ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
     }
   } else if (warp == 1) {
     // ---------------- storer ----------------
     if (lane == 0) {
-      uint32_t n = 0;
-      for (; n < my_tiles; ++n) {
+      // stages whose bulk store may still be reading them, oldest in the low bits: at most
+      // STORE_LAG + 1 stage numbers of 5 bits each
+      uint32_t pending = 0, n_pending = 0;
+      for (uint32_t n = 0; n < my_tiles; ++n) {
         const uint32_t s = n % BSR_K_BULK_STAGES, round = n / BSR_K_BULK_STAGES;
         if (!bsr_mbar_wait(bsr_smem_u32(&full_bar[s]), round & 1u, p.err_flag, &abort_flag, wait_ns)) break;
-        if (p.scatter) {
-          bsr_bulk_store(meta[s].dst, bsr_smem_u32(stage_mem + (size_t)s * BSR_K_TILE_MAX),
-                         meta[s].bytes, pol);
-          if (n >= BSR_K_BULK_STORE_LAG) {
+        const BsrStageMeta &m = meta[n % BSR_K_META_RING];
+        if (p.scatter && !m.several) {
+          bsr_bulk_store(m.dst, bsr_smem_u32(stage_mem + (size_t)s * BSR_K_TILE_MAX), m.bytes, pol);
+          pending |= s << (5u * n_pending++);
+          if (n_pending > BSR_K_BULK_STORE_LAG) {
             asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(BSR_K_BULK_STORE_LAG) : "memory");
-            bsr_mbar_arrive(bsr_smem_u32(&empty_bar[(n - BSR_K_BULK_STORE_LAG) % BSR_K_BULK_STAGES]));
+            bsr_mbar_arrive(bsr_smem_u32(&empty_bar[pending & 31u]));
+            pending >>= 5;
+            --n_pending;
           }
         } else {
+          // Nothing of this stage is the storer's to move.  Stages of earlier stores are handed back
+          // now: a lagging release waits for the next store, and none may follow for a long time,
+          // while the producer already needs those stages.
+          if (n_pending) {
+            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            for (; n_pending; --n_pending, pending >>= 5)
+              bsr_mbar_arrive(bsr_smem_u32(&empty_bar[pending & 31u]));
+          }
           bsr_mbar_arrive(bsr_smem_u32(&empty_bar[s]));
         }
       }
       if (p.scatter) {
         asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-        for (uint32_t k = (n > BSR_K_BULK_STORE_LAG ? n - BSR_K_BULK_STORE_LAG : 0); k < n; ++k)
-          bsr_mbar_arrive(bsr_smem_u32(&empty_bar[k % BSR_K_BULK_STAGES]));
+        for (; n_pending; --n_pending, pending >>= 5)
+          bsr_mbar_arrive(bsr_smem_u32(&empty_bar[pending & 31u]));
         asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // stores complete
       }
     }
@@ -432,34 +523,50 @@ bsr_install_bulk_kernel(const __grid_constant__ BsrInstallParams p) {
     // ---------------- checksum warps ----------------
     const uint32_t ct = threadIdx.x - 64;  // 0 .. 127
     uint64_t sum = 0;
-    int cur_c = -1, cur_g = -1;
+    uint32_t cur = ~0u;
     for (uint32_t n = 0; n < my_tiles; ++n) {
       const uint32_t s = n % BSR_K_BULK_STAGES, round = n / BSR_K_BULK_STAGES;
       if (!bsr_mbar_wait(bsr_smem_u32(&full_bar[s]), round & 1u, p.err_flag, &abort_flag, wait_ns)) break;
-      const BsrStageMeta m = meta[s];
-      if (m.c != cur_c || m.g != cur_g) {  // warp-uniform
-        if (cur_c >= 0) {
+      const BsrStageMeta &m = meta[n % BSR_K_META_RING];
+      const uint32_t cg = m.cg, nvec = m.bytes >> 4, word0 = m.word0;
+      if (cg != cur) {  // warp-uniform
+        if (cur != ~0u) {
           sum = bsr_warp_sum(sum);
           if (lane == 0)
-            atomicAdd((unsigned long long *)(p.acc + cur_c * BSR_K_MAX_GROUPS + cur_g),
+            atomicAdd((unsigned long long *)(p.acc + (cur >> 8) * BSR_K_MAX_GROUPS + (cur & 0xffu)),
                       (unsigned long long)sum);
         }
         sum = 0;
-        cur_c = m.c;
-        cur_g = m.g;
+        cur = cg;
       }
       const uint4 *sv = reinterpret_cast<const uint4 *>(stage_mem + (size_t)s * BSR_K_TILE_MAX);
-      const uint32_t nvec = m.bytes >> 4;
+      if (!m.several) {
 #pragma unroll 4
-      for (uint32_t v = ct; v < nvec; v += 32 * BSR_K_BULK_CONSUMER_WARPS)
-        sum += bsr_ck_vec(sv[v], m.word0 + 4u * v);
+        for (uint32_t v = ct; v < nvec; v += 32 * BSR_K_BULK_CONSUMER_WARPS)
+          sum += bsr_ck_vec(sv[v], word0 + 4u * v);
+      } else {
+        BsrRunMap rm;
+        rm.tab = m.tab;
+        rm.bases = m.bases;
+        rm.run_bytes = m.run_bytes;
+        rm.run_inv = m.run_inv;
+        rm.l0 = m.l0;
+        rm.b0 = m.b0;
+        rm.nb_shift = m.nb_shift;
+#pragma unroll 4
+        for (uint32_t v = ct; v < nvec; v += 32 * BSR_K_BULK_CONSUMER_WARPS) {
+          const uint4 w = sv[v];
+          bsr_st_stream(bsr_run_dst(rm, v), w);
+          sum += bsr_ck_vec(w, word0 + 4u * v);
+        }
+      }
       __syncwarp();
       if (lane == 0) bsr_mbar_arrive(bsr_smem_u32(&empty_bar[s]));
     }
-    if (cur_c >= 0) {
+    if (cur != ~0u) {
       sum = bsr_warp_sum(sum);
       if (lane == 0)
-        atomicAdd((unsigned long long *)(p.acc + cur_c * BSR_K_MAX_GROUPS + cur_g),
+        atomicAdd((unsigned long long *)(p.acc + (cur >> 8) * BSR_K_MAX_GROUPS + (cur & 0xffu)),
                   (unsigned long long)sum);
     }
   }

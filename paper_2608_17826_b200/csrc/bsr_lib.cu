@@ -13,6 +13,9 @@
 #include "../../include/bsr.h"
 
 #include <immintrin.h>
+#include <pthread.h>
+#include <sched.h>
+#include <sys/prctl.h>
 
 #include <atomic>
 #include <chrono>
@@ -20,6 +23,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <fstream>
 #include <memory>
 #include <mutex>
 #include <new>
@@ -38,7 +42,6 @@ using Clock = std::chrono::steady_clock;
 constexpr int kInstallThreads = 256;
 constexpr int kInstallUnroll = 2;  // 32 registers: 8 CTAs of 256 threads resident per SM
 constexpr int kLaunchSlots = 8;  // scratch sets for batched install launches in flight per restore
-constexpr uint32_t kSmCount = 148;
 constexpr uint64_t kPieceBytes = 8ull << 20;  // fill and host-to-device copy granularity
 #ifndef BSR_RING_ALLOC_FLAGS
 #define BSR_RING_ALLOC_FLAGS cudaHostAllocMapped
@@ -67,7 +70,7 @@ struct Inject {
 struct JobRes {
   cudaStream_t stream = nullptr;                        // used when the caller passes no stream
   uint8_t *dstage[BSR_MAX_RANKS] = {};                  // D staging buffers per rank
-  std::vector<cudaEvent_t> ev_h2d, ev_inst, ev_start;   // [R*D]
+  std::vector<cudaEvent_t> ev_h2d, ev_inst, ev_start;   // [n_slots]: one set per install launch in flight
   std::vector<std::pair<cudaEvent_t, cudaEvent_t>> ev_pool;  // launch timing, batched launches
   cudaEvent_t ev_done = nullptr;
   uint64_t *d_acc = nullptr;      // [n_slots][BATCH][GROUPS] checksum accumulators, kept zero
@@ -82,7 +85,8 @@ struct JobRes {
 struct StatDelta {
   uint64_t bytes_filled[BSR_MAX_RANKS] = {}, bytes_h2d[BSR_MAX_RANKS] = {},
            bytes_installed[BSR_MAX_RANKS] = {};
-  uint64_t windows = 0, kernel_launches = 0, h2d_copies = 0, install_launches = 0;
+  uint64_t windows = 0, kernel_launches = 0, h2d_copies = 0, install_launches = 0,
+           install_descriptors = 0;
   double install_kernel_ms = 0.0;
 };
 
@@ -99,6 +103,15 @@ struct Job {
   Clock::time_point t0;
   std::atomic<bool> abort{false};
   uint32_t fill_admitted = 0, fill_next = 0, fill_active = 0;  // guarded by fill_mu
+  uint64_t pieces_done = 0;     // guarded by fill_mu: fill tasks finished so far
+  std::condition_variable cv;   // with fill_mu: signalled when a fill task of this restore finishes
+};
+
+// Where the fill threads and the pinned pool are placed on a host with several NUMA nodes.
+struct NumaPlacement {
+  int node = -1;      // NUMA node of the context's GPU, -1 unknown
+  bool bind = false;  // fill threads and the allocating thread are bound to `cpus`
+  cpu_set_t cpus;
 };
 
 }  // namespace
@@ -133,6 +146,8 @@ struct bsr_req {
 struct bsr_ctx {
   bsr_config cfg{};
   uint32_t budget = 0;  // B: slots per rank shared by all restores (= W without an admission budget)
+  NumaPlacement numa;
+  uint32_t sm_count = 1;  // multiprocessors of the context's GPU: grids are sized in whole waves of it
   std::mutex mu, restore_mu, aux_mu, setup_mu, fill_mu, pool_mu;
   std::string err;
 
@@ -146,6 +161,7 @@ struct bsr_ctx {
   uint32_t pieces = 1;  // fill pieces per chunk
   std::atomic<bool> finalized{false};
   bool use_bulk = true;  // the install kernel chosen for this registration (see finalize_registration)
+  bool has_spans = false;  // the tile table holds spans of several runs
   std::vector<BsrTile> h_tiles;
   BsrTile *d_tiles = nullptr;
   uint64_t *d_tensor_base = nullptr;
@@ -224,6 +240,7 @@ void merge_stats(bsr_ctx *c, const StatDelta &d) {
   c->st.kernel_launches += d.kernel_launches;
   c->st.h2d_copies += d.h2d_copies;
   c->st.install_launches += d.install_launches;
+  c->st.install_descriptors += d.install_descriptors;
   c->st.install_kernel_ms += d.install_kernel_ms;
 }
 
@@ -237,30 +254,63 @@ int finalize_registration(bsr_ctx *c) {
   std::vector<uint32_t> tgroup(c->L), trun(c->L);
   uint64_t off = 0;
   c->h_tiles.clear();
-  for (uint32_t l = 0; l < c->L; ++l) {
+  for (uint32_t l = 0; l < c->L;) {
     const TensorReg &t = c->tensors[l];
     const uint32_t B = c->groups[t.group].block_tokens;
     const uint32_t nb = BSR_CHUNK_TOKENS / B;
     const uint64_t run = (uint64_t)B * t.bytes_per_token;
-    tgroup[l] = t.group;
-    trun[l] = (uint32_t)run;
-    const uint32_t nsplit = (uint32_t)((run + BSR_K_TILE_MAX - 1) / BSR_K_TILE_MAX);
-    const uint32_t piece = (uint32_t)round_up((run + nsplit - 1) / nsplit, 128);
-    for (uint32_t b = 0; b < nb; ++b) {
-      for (uint64_t s = 0; s < run; s += piece) {
-        BsrTile tl{};
-        tl.src_off = (uint32_t)(off + b * run + s);
-        tl.bytes = (uint32_t)((run - s < piece) ? run - s : piece);
-        tl.dst_off = (uint32_t)s;
+    const uint32_t run_inv = (uint32_t)(((1ull << 32) + run - 1) / run);
+    // a family: this tensor and the ones after it with the same group and bytes per token; their
+    // runs have one length and lie back to back in the chunk
+    // Runs of up to BSR_K_SPAN_RUN_MAX bytes travel several to a span: below that a bulk copy per
+    // run costs more in issue and stage turnover (about 150 ns per CTA) than its bytes are worth.
+    const bool spans = run <= BSR_K_SPAN_RUN_MAX && 2 * run <= BSR_K_TILE_MAX;
+    uint32_t l_end = l + 1;
+    if (spans)
+      while (l_end < c->L && c->tensors[l_end].group == t.group &&
+             c->tensors[l_end].bytes_per_token == t.bytes_per_token)
+        ++l_end;
+    for (uint32_t k = l; k < l_end; ++k) {
+      tgroup[k] = t.group;
+      trun[k] = (uint32_t)run;
+    }
+    BsrTile tl{};
+    tl.run_bytes = (uint32_t)run;
+    tl.run_inv = run_inv;
+    tl.group = (uint8_t)t.group;
+    if (spans) {
+      // short runs: spans of as many whole runs as a stage holds, across the family's tensors
+      const uint32_t per_span = (uint32_t)(BSR_K_TILE_MAX / run);
+      const uint32_t runs = (l_end - l) * nb;
+      for (uint32_t v0 = 0; v0 < runs; v0 += per_span) {
+        const uint32_t cnt = runs - v0 < per_span ? runs - v0 : per_span;
+        tl.src_off = (uint32_t)(off + (uint64_t)v0 * run);
+        tl.bytes = (uint32_t)(cnt * run);
+        tl.dst_off = 0;
         tl.word0 = (uint32_t)((tl.src_off - c->seg_begin[t.group]) / 4);
-        tl.run_bytes = (uint32_t)run;
-        tl.tensor = (uint16_t)l;
-        tl.group = (uint8_t)t.group;
-        tl.blk = (uint8_t)b;
+        tl.tensor = (uint16_t)(l + v0 / nb);
+        tl.blk = (uint8_t)(v0 % nb);
+        tl.n_runs = cnt;
         c->h_tiles.push_back(tl);
       }
+    } else {
+      // long runs: each run on its own, cut into pieces of at most a stage
+      const uint32_t nsplit = (uint32_t)((run + BSR_K_TILE_MAX - 1) / BSR_K_TILE_MAX);
+      const uint32_t piece = (uint32_t)round_up((run + nsplit - 1) / nsplit, 128);
+      for (uint32_t b = 0; b < nb; ++b)
+        for (uint64_t s = 0; s < run; s += piece) {
+          tl.src_off = (uint32_t)(off + b * run + s);
+          tl.bytes = (uint32_t)((run - s < piece) ? run - s : piece);
+          tl.dst_off = (uint32_t)s;
+          tl.word0 = (uint32_t)((tl.src_off - c->seg_begin[t.group]) / 4);
+          tl.tensor = (uint16_t)l;
+          tl.blk = (uint8_t)b;
+          tl.n_runs = 1;
+          c->h_tiles.push_back(tl);
+        }
     }
-    off += (uint64_t)BSR_CHUNK_TOKENS * t.bytes_per_token;
+    off += (uint64_t)(l_end - l) * BSR_CHUNK_TOKENS * t.bytes_per_token;
+    l = l_end;
   }
   // the kernels count the tiles of a launch (up to BSR_K_MAX_BATCH chunks) in 32 bits
   if (c->h_tiles.size() > (1u << 22))
@@ -284,11 +334,19 @@ int finalize_registration(bsr_ctx *c) {
     std::lock_guard<std::mutex> g(c->mu);
     c->st.dev_aux_bytes += c->h_tiles.size() * sizeof(BsrTile) + bases.size() * 8 + c->L * 8;
   }
-  // Kernel choice.  Measured on B200 with both kernels launched in several waves: the bulk-copy
-  // kernel is level with the vector kernel where nearly all bytes sit in long tiles (1.276 against
-  // 1.283 ms per 256-descriptor launch) and 8 % ahead with many short runs, where most of a
-  // 256-thread CTA of the vector kernel idles.  So BSR_INSTALL_AUTO means the bulk-copy kernel.
-  c->use_bulk = c->cfg.install_variant != BSR_INSTALL_VECTOR;
+  // Kernel choice.  Measured on B200, 256-descriptor launches: where most bytes sit in runs that
+  // travel on their own the bulk-copy kernel runs at the speed of a device copy (1.28 ms on the
+  // baseline registration; the vector kernel needs full occupancy to come within 5 % of it).  Where
+  // most bytes sit in short runs, moved as spans of several runs, every store is a 16-byte vector
+  // store in either kernel, and the vector kernel has sixteen times the warps to issue them with
+  // (0.89 against 0.76 of the copy rate on a registration of 256-byte runs).
+  uint64_t span_bytes = 0;
+  for (const BsrTile &tl : c->h_tiles)
+    if (tl.n_runs > 1) span_bytes += tl.bytes;
+  c->has_spans = span_bytes != 0;
+  const bool mostly_short_runs = 2 * span_bytes > c->chunk_bytes;
+  c->use_bulk = c->cfg.install_variant == BSR_INSTALL_BULK ||
+                (c->cfg.install_variant == BSR_INSTALL_AUTO && !mostly_short_runs);
   c->finalized.store(true, std::memory_order_release);
   return BSR_OK;
 }
@@ -321,24 +379,31 @@ int launch_install(bsr_ctx *c, const BsrInstallParams &p, cudaStream_t s, StatDe
     // Whole waves of the CTAs an SM holds, each CTA streaming BSR_K_BULK_TILES_PER_CTA tiles through
     // its stage ring: several waves instead of one persistent wave let the hardware scheduler even
     // out the tail (measured on B200: 1.28 ms against 1.35 ms per 256-descriptor launch).
-    const uint64_t wave = (uint64_t)kSmCount * BSR_K_BULK_CTAS_PER_SM;
+    const uint64_t wave = (uint64_t)c->sm_count * BSR_K_BULK_CTAS_PER_SM;
     uint64_t want = (total / BSR_K_BULK_TILES_PER_CTA + wave - 1) / wave * wave;
     if (want < wave) want = wave;
+#ifdef BSR_K_BULK_MAX_GRID  // test builds: few CTAs, so that each one cycles its stage ring many times
+    if (want > BSR_K_BULK_MAX_GRID) want = BSR_K_BULK_MAX_GRID;
+#endif
     bsr_install_bulk_kernel<<<(uint32_t)(total < want ? total : want), BSR_K_BULK_THREADS,
                               BSR_K_BULK_SMEM, s>>>(p);
   } else {
     // About nine tiles per CTA, in whole waves of the 8 CTAs an SM holds: many more CTAs than are
     // resident let the hardware scheduler even out the tail (measured best on B200; one tile per
     // CTA and a single persistent wave are both slower).
-    const uint64_t wave = (uint64_t)kSmCount * 8;
+    const uint64_t wave = (uint64_t)c->sm_count * 8;
     uint64_t want = (total / 9 + wave - 1) / wave * wave;
     if (want < 2 * wave) want = 2 * wave;
-    bsr_install_vec_kernel<kInstallThreads, kInstallUnroll>
-        <<<(uint32_t)(total < want ? total : want), kInstallThreads, 0, s>>>(p);
+    const uint32_t grid = (uint32_t)(total < want ? total : want);
+    if (c->has_spans)
+      bsr_install_vec_kernel<kInstallThreads, kInstallUnroll, true><<<grid, kInstallThreads, 0, s>>>(p);
+    else
+      bsr_install_vec_kernel<kInstallThreads, kInstallUnroll, false><<<grid, kInstallThreads, 0, s>>>(p);
   }
   CU(c, cudaGetLastError());
   sd.kernel_launches++;
   sd.install_launches++;
+  sd.install_descriptors += p.n_chunks;
   return BSR_OK;
 }
 
@@ -403,10 +468,10 @@ int acquire_res(bsr_ctx *c, JobRes **out) {
     std::lock_guard<std::mutex> g(c->mu);
     c->st.dev_aux_bytes += (uint64_t)R * D * c->chunk_bytes;
   }
-  res->ev_h2d.resize(R * D);
-  res->ev_inst.resize(R * D);
-  res->ev_start.resize(R * D);
-  for (uint32_t k = 0; k < R * D; ++k) {
+  res->ev_h2d.resize(res->n_slots);
+  res->ev_inst.resize(res->n_slots);
+  res->ev_start.resize(res->n_slots);
+  for (uint32_t k = 0; k < res->n_slots; ++k) {
     CU(c, cudaEventCreateWithFlags(&res->ev_h2d[k], cudaEventDisableTiming));
     CU(c, cudaEventCreate(&res->ev_inst[k]));
     CU(c, cudaEventCreate(&res->ev_start[k]));
@@ -456,6 +521,7 @@ void fill_copy(uint8_t *dst, const uint8_t *src, size_t n) {
 // let the first device copy start after a fraction of a chunk has been fetched and keep all threads
 // busy on the chunks the copy engine needs next.  Restores in flight are served round-robin.
 void filler_main(bsr_ctx *c) {
+  if (c->numa.bind) pthread_setaffinity_np(pthread_self(), sizeof(cpu_set_t), &c->numa.cpus);
   for (;;) {
     Job *job = nullptr;
     uint32_t t = 0;
@@ -538,11 +604,70 @@ void filler_main(bsr_ctx *c) {
     job->t_piece[t] = (uint64_t)std::chrono::duration_cast<std::chrono::nanoseconds>(Clock::now() - job->t0).count();
     job->state[t].store(state, std::memory_order_release);
     {
+      // the restore thread sleeps on job->cv; it is signalled under the lock because the Job lives
+      // on that thread's stack and may go away as soon as fill_active reaches zero
       std::lock_guard<std::mutex> lk(c->fill_mu);
       job->fill_active--;
+      job->pieces_done++;
+      job->cv.notify_one();
     }
     c->fill_cv.notify_all();
   }
+}
+
+// ---- host placement ---------------------------------------------------------------------------
+// "0-3,8,10-11" -> CPU set.  Returns the number of CPUs named, -1 on a malformed list.
+int parse_cpulist(const char *s, cpu_set_t *set) {
+  CPU_ZERO(set);
+  int n = 0;
+  const char *p = s;
+  while (*p && *p != '\n') {
+    char *end = nullptr;
+    const long lo = strtol(p, &end, 10);
+    if (end == p || lo < 0) return -1;
+    long hi = lo;
+    p = end;
+    if (*p == '-') {
+      hi = strtol(p + 1, &end, 10);
+      if (end == p + 1 || hi < lo) return -1;
+      p = end;
+    }
+    for (long k = lo; k <= hi; ++k)
+      if (k < CPU_SETSIZE) {
+        CPU_SET((int)k, set);
+        ++n;
+      }
+    if (*p == ',') ++p;
+  }
+  return n;
+}
+
+bool read_line(const std::string &path, std::string *out) {
+  std::ifstream f(path);
+  if (!f) return false;
+  std::getline(f, *out);
+  return true;
+}
+
+// Decides where this context's fill threads and pinned pool go (see bsr_config.numa_bind).
+void plan_numa(bsr_ctx *c) {
+  CPU_ZERO(&c->numa.cpus);
+  if (c->cfg.numa_bind == BSR_NUMA_OFF) return;
+  char bus[32] = {};
+  if (cudaDeviceGetPCIBusId(bus, sizeof bus, c->cfg.device) != cudaSuccess) {
+    cudaGetLastError();
+    return;
+  }
+  int node = -1, n_nodes = 0;
+  char list[1024] = {};
+  if (bsr_numa_of_pci("/sys", bus, &node, list, sizeof list, &n_nodes) != BSR_OK) return;
+  c->numa.node = node;
+  if (node < 0 || (n_nodes < 2 && c->cfg.numa_bind != BSR_NUMA_ALWAYS)) return;
+  cpu_set_t want, have;
+  if (parse_cpulist(list, &want) <= 0) return;
+  if (sched_getaffinity(0, sizeof have, &have) != 0) return;
+  CPU_AND(&c->numa.cpus, &want, &have);  // never widen what the process was given
+  c->numa.bind = CPU_COUNT(&c->numa.cpus) > 0;
 }
 
 // The pinned slot pool: B slots per rank (B = W unless an admission budget is configured).
@@ -551,14 +676,32 @@ int ensure_ring(bsr_ctx *c) {
   std::lock_guard<std::mutex> sl(c->setup_mu);
   if (c->ring_ready.load(std::memory_order_acquire)) return BSR_OK;
   const uint32_t R = c->cfg.n_ranks, B = c->budget;
-  for (uint32_t r = 0; r < R; ++r) {
-    if (cudaHostAlloc((void **)&c->ring[r], (size_t)B * c->slot_bytes, BSR_RING_ALLOC_FLAGS) !=
-            cudaSuccess ||
-        cudaHostGetDevicePointer((void **)&c->ring_dev[r], c->ring[r], 0) != cudaSuccess) {
-      cudaGetLastError();
-      return fail(c, BSR_ERR_NOMEM, "pinned pool of %u x %llu bytes", B,
-                  (unsigned long long)c->slot_bytes);
+  // Pinned pages are placed where the allocating thread runs: on a host with several NUMA nodes
+  // the pool is allocated from a thread bound to the GPU's node, so that neither the fill threads
+  // (bound to the same node) nor the GPU's DMA reads cross the socket interconnect.
+  int alloc_rc = BSR_OK;
+  auto alloc = [&] {
+    if (c->numa.bind) pthread_setaffinity_np(pthread_self(), sizeof(cpu_set_t), &c->numa.cpus);
+    if (cudaSetDevice(c->cfg.device) != cudaSuccess) {
+      alloc_rc = BSR_ERR_CUDA;
+      return;
     }
+    for (uint32_t r = 0; r < R; ++r)
+      if (cudaHostAlloc((void **)&c->ring[r], (size_t)B * c->slot_bytes, BSR_RING_ALLOC_FLAGS) !=
+              cudaSuccess ||
+          cudaHostGetDevicePointer((void **)&c->ring_dev[r], c->ring[r], 0) != cudaSuccess) {
+        cudaGetLastError();
+        alloc_rc = BSR_ERR_NOMEM;
+        return;
+      }
+  };
+  if (c->numa.bind)
+    std::thread(alloc).join();
+  else
+    alloc();
+  if (alloc_rc != BSR_OK)
+    return fail(c, alloc_rc, "pinned pool of %u x %llu bytes", B, (unsigned long long)c->slot_bytes);
+  for (uint32_t r = 0; r < R; ++r) {
     {
       std::lock_guard<std::mutex> g(c->mu);
       c->st.ring_bytes_allocated[r] = (uint64_t)B * c->slot_bytes;
@@ -676,14 +819,34 @@ int restore_resident(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
 }
 
 // ---- restore through the pinned slot pool --------------------------------------------------------
+// `stages` selects how much of the pipeline runs: everything (a restore), or, for calibration, only
+// the fill (tier -> slot) or the fill plus the copies to device staging.  The calibration forms
+// take the same slots in the same order with the same threads but launch no kernel, so they touch
+// neither the paged cache nor the request's bitmap.
+enum { kStagesAll = 0, kStagesFill = BSR_CAL_FILL, kStagesFillH2d = BSR_CAL_FILL_H2D };
+
 int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
-                 Clock::time_point deadline, StatDelta &sd) {
+                 Clock::time_point deadline, StatDelta &sd, int stages = kStagesAll) {
   int rc = ensure_ring(c);
   if (rc != BSR_OK) return rc;
   const uint32_t R = c->cfg.n_ranks, W = c->cfg.window_chunks, D = c->cfg.dev_staging_depth;
   const uint32_t N = q->n_adv, total = N * R;
   const uint32_t P = c->pieces;
-  const bool direct = c->cfg.direct_install != 0;
+  const bool direct = c->cfg.direct_install != 0 && stages == kStagesAll;
+  const uint32_t n_ev = res->n_slots;  // launch slots: a scratch set and three events each
+  // Chunks of each rank that one install launch takes.  A launch costs about 13 us on top of its
+  // bytes (25 us while the copy engine is busy, which here it always is), so a single 16 MB chunk
+  // (5 us of traffic) runs at a fraction of device-copy speed and 16 chunks at three quarters of
+  // it; fewer chunks per launch hand the window's slots back sooner.  A launch never needs more
+  // staging buffers than a rank has, and leaves three quarters of the window to the fill.
+  uint32_t cpl = c->cfg.install_batch / R;
+  if (cpl > D) cpl = D;
+  if (cpl > W / 4) cpl = W / 4;
+  if (cpl > BSR_K_MAX_BATCH / R) cpl = BSR_K_MAX_BATCH / R;
+  if (cpl == 0) cpl = 1;
+  // items (chunk, rank) per launch; a kernel that reads pinned slots over the link takes one
+  const uint32_t gsz = direct ? 1 : cpl * R;
+
   Job job;
   job.q = q;
   job.deadline = deadline;
@@ -702,14 +865,25 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
     std::lock_guard<std::mutex> lk(c->fill_mu);
     c->jobs.push_back(&job);
   }
-  uint32_t admitted = 0, submitted = 0, reaped = 0, cur_piece = 0;
+  // items are numbered s = i * R + r in admission order; each counter below is a prefix length
+  uint32_t admitted = 0, submitted = 0, launched = 0, reaped = 0, cur_piece = 0;
+  struct Launch {
+    uint32_t first, count;
+  };
+  std::vector<Launch> launches;                // install launches issued, in order
+  size_t launches_reaped = 0;                  // ... of which observed complete
+  std::vector<int64_t> buf_launch(R * D, -1);  // the launch that last read each staging buffer
   uint32_t live[BSR_MAX_RANKS] = {};
+  uint64_t seen_done = 0;
   Inject inj;
   {
     std::lock_guard<std::mutex> lk(c->mu);
     inj = c->inject;
   }
   bool stop = false;  // a failure was seen: admit and submit nothing more, drain
+  // short sleeps while polling events: without this the kernel rounds them up by 50 us
+  const int slack_before = prctl(PR_GET_TIMERSLACK);
+  prctl(PR_SET_TIMERSLACK, 1000UL);
 
   auto first_error = [&](int code) {
     if (rc == BSR_OK) rc = code;
@@ -721,6 +895,64 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
     std::lock_guard<std::mutex> pl(c->pool_mu);
     c->free_slots[r].push_back(job.slot[s]);
     c->live_total[r]--;
+  };
+  // Closes the open group [launched, submitted): one install launch over all its descriptors.
+  auto launch_group = [&]() {
+    const uint32_t first = launched, n = submitted - launched;
+    const size_t li = launches.size();
+    const uint32_t ls = (uint32_t)(li % n_ev);
+    cudaError_t e = cudaSuccess;
+    if (stages == kStagesFill) {
+      // nothing was queued on the GPU: the group counts as complete at once
+    } else if (stages == kStagesFillH2d) {
+      e = cudaEventRecord(res->ev_inst[ls], c->copy_stream);
+    } else {
+      if (!direct) {
+        e = cudaEventRecord(res->ev_h2d[ls], c->copy_stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, res->ev_h2d[ls], 0);
+      }
+      BsrInstallParams p{};
+      fill_params(c, p, res, ls);
+      p.n_adv = N;
+      p.scatter = 1;
+      p.tables = q->d_table_ptrs;
+      p.ck_out = q->d_ck;
+      p.verdict = q->d_verdict;
+      p.n_chunks = n;
+      bool host_source = false;
+      if (n == 1) {
+        p.one = q->h_desc[first];  // carried in the kernel parameters
+        host_source = direct && job.objs[first].loc == BSR_LOC_HOST;
+      } else {
+        p.batch = q->d_desc + first;
+        if (e == cudaSuccess)
+          e = cudaMemcpyAsync(q->d_desc + first, q->h_desc + first, (size_t)n * sizeof(BsrChunkDesc),
+                              cudaMemcpyHostToDevice, stream);
+      }
+      for (uint32_t s = first; s < first + n; ++s)
+        if (inj.kind == BSR_INJECT_KERNEL_WAIT && inj.rank == s % R && inj.chunk == s / R) {
+          p.stall_tile = 0;             // the first tile of this launch is never loaded ...
+          p.wait_ns = 50ull * 1000000;  // ... and every wait in the kernel gives up after 50 ms
+        }
+      if (e == cudaSuccess && c->cfg.time_kernels) e = cudaEventRecord(res->ev_start[ls], stream);
+      if (e != cudaSuccess) {
+        first_error(fail(c, BSR_ERR_TRANSFER, "install submit: %s", cudaGetErrorString(e)));
+        return;
+      }
+      const int lrc = launch_install(c, p, stream, sd, host_source);
+      e = cudaEventRecord(res->ev_inst[ls], stream);
+      if (lrc != BSR_OK) {
+        first_error(lrc);
+        return;
+      }
+    }
+    if (e != cudaSuccess) {
+      first_error(fail(c, BSR_ERR_CUDA, "record: %s", cudaGetErrorString(e)));
+      return;
+    }
+    for (uint32_t s = first; s < first + n; ++s) buf_launch[(s % R) * D + (s / R) % D] = (int64_t)li;
+    launches.push_back(Launch{first, n});
+    launched = submitted;
   };
 
   while (true) {
@@ -758,35 +990,42 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
         progress = true;
       }
     }
-    // reap, in order: observe the install of the oldest chunk in flight, release its slot
-    while (reaped < submitted) {
-      const uint32_t i = reaped / R, r = reaped % R, k = r * D + i % D;
-      cudaError_t e = cudaEventQuery(res->ev_inst[k]);
+    // reap, in order: observe the oldest install launch in flight, release the slots of its chunks
+    while (launches_reaped < launches.size()) {
+      const Launch &L = launches[launches_reaped];
+      const uint32_t ls = (uint32_t)(launches_reaped % n_ev);
+      cudaError_t e = stages == kStagesFill ? cudaSuccess : cudaEventQuery(res->ev_inst[ls]);
       if (e == cudaErrorNotReady) break;
       if (e != cudaSuccess) {
         first_error(fail(c, BSR_ERR_CUDA, "install event: %s", cudaGetErrorString(e)));
-        while (reaped < submitted) {  // the context is unusable; nothing more can be observed
+        while (reaped < launched) {  // the context is unusable; nothing more can be observed
           release_slot(reaped);
           live[reaped % R]--;
           ++reaped;
         }
+        launches_reaped = launches.size();
         break;
       }
-      if (c->cfg.time_kernels) {
+      if (c->cfg.time_kernels && stages == kStagesAll) {
         float ms = 0.f;
-        if (cudaEventElapsedTime(&ms, res->ev_start[k], res->ev_inst[k]) == cudaSuccess)
+        if (cudaEventElapsedTime(&ms, res->ev_start[ls], res->ev_inst[ls]) == cudaSuccess)
           sd.install_kernel_ms += ms;
       }
-      const int h = harvest(c, q, r, i, sd);
-      if (h != BSR_OK) first_error(h);
-      job.trace[reaped].t_done_ns = now_ns();
-      release_slot(reaped);
-      live[r]--;
-      ++reaped;
+      for (uint32_t s = L.first; s < L.first + L.count; ++s) {
+        if (stages == kStagesAll) {
+          const int h = harvest(c, q, s % R, s / R, sd);
+          if (h != BSR_OK) first_error(h);
+        }
+        job.trace[s].t_done_ns = now_ns();
+        release_slot(s);
+        live[s % R]--;
+      }
+      reaped = L.first + L.count;
+      ++launches_reaped;
       progress = true;
     }
-    // submit, in order: every ready piece slot -> device staging on the copy stream; when the chunk
-    // is complete, the install kernel on the compute stream
+    // submit, in order: every ready piece slot -> device staging on the copy stream; a chunk whose
+    // pieces are all queued joins the open group, and a full group is launched
     while (!stop && submitted < admitted && submitted - reaped < R * D) {
       const uint32_t i = submitted / R, r = submitted % R, d = i % D, k = r * D + d;
       uint8_t *stage = direct ? nullptr : res->dstage[r] + (size_t)d * c->chunk_bytes;
@@ -807,8 +1046,10 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
         const uint64_t off = (uint64_t)cur_piece * kPieceBytes;
         const uint64_t len = (c->chunk_bytes - off < kPieceBytes) ? c->chunk_bytes - off : kPieceBytes;
         const uint8_t *from = (o.loc == BSR_LOC_HOST) ? slot_host + off : o.data + off;
-        if (!direct) {
-          if (cur_piece == 0) e = cudaStreamWaitEvent(c->copy_stream, res->ev_inst[k], 0);
+        if (!direct && stages != kStagesFill) {
+          // the staging buffer is free once the install launch that last read it has finished
+          if (cur_piece == 0 && stages == kStagesAll && buf_launch[k] >= (int64_t)launches_reaped)
+            e = cudaStreamWaitEvent(c->copy_stream, res->ev_inst[buf_launch[k] % n_ev], 0);
           if (e == cudaSuccess)
             e = cudaMemcpyAsync(stage + off, from, len, cudaMemcpyDefault, c->copy_stream);
           if (e != cudaSuccess) {
@@ -818,47 +1059,22 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
           sd.h2d_copies++;
         }
         sd.bytes_filled[r] += (o.loc == BSR_LOC_HOST) ? len : 0;
-        sd.bytes_h2d[r] += len;  // bytes that cross the host link, by copy or by kernel loads
+        if (stages != kStagesFill)
+          sd.bytes_h2d[r] += len;  // bytes that cross the host link, by copy or by kernel loads
         ++cur_piece;
         progress = true;
       }
       if (stop || blocked) break;
       const TierObj &o = job.objs[submitted];
-      if (!direct) {
-        e = cudaEventRecord(res->ev_h2d[k], c->copy_stream);
-        if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, res->ev_h2d[k], 0);
-      }
-      if (e == cudaSuccess && c->cfg.time_kernels) e = cudaEventRecord(res->ev_start[k], stream);
-      if (e != cudaSuccess) {
-        first_error(fail(c, BSR_ERR_TRANSFER, "copy submit: %s", cudaGetErrorString(e)));
-        break;
-      }
-      BsrInstallParams p{};
-      fill_params(c, p, res, k);
-      p.n_adv = N;
-      p.scatter = 1;
-      p.tables = q->d_table_ptrs;
-      p.ck_out = q->d_ck;
-      p.verdict = q->d_verdict;
-      p.n_chunks = 1;
+      BsrChunkDesc &cd = q->h_desc[submitted];
       // direct mode: the kernel reads the pinned slot (or the device object) itself over the link
-      p.one.src = !direct ? stage
-                          : (o.loc == BSR_LOC_HOST
-                                 ? c->ring_dev[r] + (size_t)job.slot[submitted] * c->slot_bytes
-                                 : o.data);
-      p.one.chunk = i;
-      p.one.rank = r;
-      for (uint32_t g = 0; g < c->G; ++g) p.one.expect[g] = o.ck[g];
-      if (inj.kind == BSR_INJECT_KERNEL_WAIT && inj.rank == r && inj.chunk == i) {
-        p.stall_tile = 0;            // the first tile of this launch is never loaded ...
-        p.wait_ns = 50ull * 1000000;  // ... and every wait in the kernel gives up after 50 ms
-      }
-      const int lrc = launch_install(c, p, stream, sd, direct && o.loc == BSR_LOC_HOST);
-      e = cudaEventRecord(res->ev_inst[k], stream);
-      if (lrc != BSR_OK || e != cudaSuccess) {
-        first_error(lrc != BSR_OK ? lrc : fail(c, BSR_ERR_CUDA, "record: %s", cudaGetErrorString(e)));
-        break;
-      }
+      cd.src = !direct ? stage
+                       : (o.loc == BSR_LOC_HOST
+                              ? c->ring_dev[r] + (size_t)job.slot[submitted] * c->slot_bytes
+                              : o.data);
+      cd.chunk = i;
+      cd.rank = r;
+      for (uint32_t g = 0; g < BSR_MAX_GROUPS; ++g) cd.expect[g] = g < c->G ? o.ck[g] : 0;
       for (uint32_t pc = 0; pc < P; ++pc)
         if (job.t_piece[(size_t)submitted * P + pc] > job.trace[submitted].t_filled_ns)
           job.trace[submitted].t_filled_ns = job.t_piece[(size_t)submitted * P + pc];
@@ -866,8 +1082,9 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
       ++submitted;
       cur_piece = 0;
       progress = true;
+      if (submitted - launched == gsz || submitted == total) launch_group();
     }
-    if (reaped == submitted && (stop || reaped == total)) break;
+    if (reaped == launched && launches_reaped == launches.size() && (stop || reaped == total)) break;
     if (!progress) {
       if (Clock::now() > deadline) {
         first_error(BSR_ERR_TIMEOUT);
@@ -876,11 +1093,26 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
         cudaStreamSynchronize(stream);
         continue;
       }
-      std::this_thread::yield();
+      // A group that cannot grow must not wait to be full: every admitted chunk has been queued,
+      // nothing is in flight whose completion would free a slot, and admission is held up (the
+      // window is full, or other restores hold the rest of the pool).
+      if (!stop && submitted > launched && submitted == admitted && cur_piece == 0 &&
+          launches_reaped == launches.size()) {
+        launch_group();
+        continue;
+      }
+      // Sleep until a fill task of this restore finishes, or for a short while when there is an
+      // event to poll (the fill threads need the cores more than a spinning waiter does).
+      std::unique_lock<std::mutex> lk(c->fill_mu);
+      if (job.pieces_done == seen_done)
+        job.cv.wait_for(lk, launches_reaped < launches.size() ? std::chrono::microseconds(20)
+                                                              : std::chrono::microseconds(200));
+      seen_done = job.pieces_done;
     }
   }
-  // copies of a chunk that never reached its install launch may still be queued
-  if (cur_piece != 0) cudaStreamSynchronize(c->copy_stream);
+  prctl(PR_SET_TIMERSLACK, slack_before > 0 ? (unsigned long)slack_before : 0UL);
+  // copies of chunks that never reached an install launch may still be queued
+  if (submitted > launched || cur_piece != 0) cudaStreamSynchronize(c->copy_stream);
   // quiesce the fillers: nothing of this request may be touched after return
   job.abort.store(true, std::memory_order_release);
   {
@@ -1022,12 +1254,16 @@ int bsr_ctx_create(const bsr_config *cfg, bsr_ctx **out) {
     c->cfg.load_concurrency = hw < 4 ? 4 : (hw > 16 ? 16 : hw);
   }
   if (c->cfg.load_concurrency > 64) c->cfg.load_concurrency = 64;
-  if (c->cfg.dev_staging_depth == 0) c->cfg.dev_staging_depth = 4;
+  if (c->cfg.dev_staging_depth == 0) c->cfg.dev_staging_depth = 12;
+  if (c->cfg.install_batch == 0) c->cfg.install_batch = 16;
   if (c->cfg.dev_staging_depth > 16) c->cfg.dev_staging_depth = 16;
   if (c->cfg.timeout_ms == 0) c->cfg.timeout_ms = 30000;
   if (c->cfg.slot_align == 0) c->cfg.slot_align = 4096;
   c->budget = c->cfg.budget_slots ? c->cfg.budget_slots : c->cfg.window_chunks;
+  int sms = 0;
   bool ok = cudaSetDevice(cfg->device) == cudaSuccess &&
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device) == cudaSuccess &&
+            sms > 0 &&
             cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess &&
             cudaStreamCreateWithFlags(&c->own_stream, cudaStreamNonBlocking) == cudaSuccess &&
             init_scratch(c, &c->aux, kLaunchSlots) == BSR_OK &&
@@ -1039,6 +1275,9 @@ int bsr_ctx_create(const bsr_config *cfg, bsr_ctx **out) {
     bsr_ctx_destroy(c);
     return BSR_ERR_CUDA;
   }
+  c->sm_count = (uint32_t)sms;
+  plan_numa(c);
+  c->st.fill_numa_node = c->numa.bind ? c->numa.node : -1;
   *out = c;
   return BSR_OK;
 }
@@ -1078,7 +1317,15 @@ int bsr_ctx_destroy(bsr_ctx *c) {
   return BSR_OK;
 }
 
-const char *bsr_last_error(bsr_ctx *c) { return c ? c->err.c_str() : "null context"; }
+const char *bsr_last_error(bsr_ctx *c) {
+  // A copy per calling thread: a failing call on another thread may replace the context's text at
+  // any time, so the context's own buffer is never handed out.
+  static thread_local std::string mine;
+  if (!c) return "null context";
+  std::lock_guard<std::mutex> lk(c->mu);
+  mine = c->err;
+  return mine.c_str();
+}
 
 int bsr_register(bsr_ctx *c, uint32_t rank, const bsr_group_desc *groups, uint32_t n_groups,
                  const bsr_tensor_desc *tensors, uint32_t n_tensors) {
@@ -1104,6 +1351,14 @@ int bsr_register(bsr_ctx *c, uint32_t rank, const bsr_group_desc *groups, uint32
     if (!t.dev_base || (reinterpret_cast<uintptr_t>(t.dev_base) & 15u))
       return fail(c, BSR_ERR_ALIGN, "tensor %u: dev_base must be 16-byte aligned", l);
     per_token += t.bytes_per_token;
+  }
+  // every group owns at least one tensor: an empty segment would "verify" as 0 == 0 and count
+  // toward the commit predicate without any byte behind it
+  {
+    bool owned[BSR_MAX_GROUPS] = {};
+    for (uint32_t l = 0; l < n_tensors; ++l) owned[tensors[l].group] = true;
+    for (uint32_t g = 0; g < n_groups; ++g)
+      if (!owned[g]) return fail(c, BSR_ERR_INVALID, "group %u has no tensor", g);
   }
   if (per_token * BSR_CHUNK_TOKENS >= (1ull << 32))
     return fail(c, BSR_ERR_INVALID, "chunk larger than 4 GiB");
@@ -1482,6 +1737,66 @@ int bsr_restore(bsr_ctx *c, bsr_req *q, void *cuda_stream) {
   return rc;
 }
 
+int bsr_restore_calibrate(bsr_ctx *c, bsr_req *q, int stages, double *seconds) {
+  if (!c || !q || q->ctx != c || !seconds || (stages != BSR_CAL_FILL && stages != BSR_CAL_FILL_H2D))
+    return BSR_ERR_INVALID;
+  join_async(q);
+  std::lock_guard<std::mutex> ql(q->mu);
+  std::unique_lock<std::mutex> serial(c->restore_mu, std::defer_lock);
+  if (c->cfg.budget_slots == 0) serial.lock();
+  *seconds = 0.0;
+  if (q->n_adv == 0) return BSR_OK;
+  CU(c, cudaSetDevice(c->cfg.device));
+  JobRes *res = nullptr;
+  int rc = acquire_res(c, &res);
+  if (rc != BSR_OK) {
+    if (res) release_res(c, res);
+    return rc;
+  }
+  StatDelta sd;  // discarded: a calibration pass is not a restore
+  const auto t0 = Clock::now();
+  rc = restore_ring(c, q, res, res->stream, t0 + std::chrono::milliseconds(c->cfg.timeout_ms), sd,
+                    stages);
+  cudaStreamSynchronize(c->copy_stream);
+  *seconds = std::chrono::duration<double>(Clock::now() - t0).count();
+  release_res(c, res);
+  return rc;
+}
+
+int bsr_numa_of_pci(const char *sysfs_root, const char *pci_bus_id, int *node, char *cpulist,
+                    size_t cpulist_cap, int *n_nodes) {
+  if (!sysfs_root || !pci_bus_id || !node) return BSR_ERR_INVALID;
+  std::string id(pci_bus_id);
+  for (char &ch : id)
+    if (ch >= 'A' && ch <= 'F') ch = (char)(ch - 'A' + 'a');  // sysfs spells bus ids in lower case
+  const std::string root(sysfs_root);
+  std::string line;
+  if (!read_line(root + "/bus/pci/devices/" + id + "/numa_node", &line)) return BSR_ERR_MISSING;
+  char *end = nullptr;
+  const long v = strtol(line.c_str(), &end, 10);
+  if (end == line.c_str()) return BSR_ERR_INVALID;
+  *node = (int)v;
+  int count = 0;
+  for (int k = 0; k < 1024; ++k) {
+    std::string dummy;
+    if (!read_line(root + "/devices/system/node/node" + std::to_string(k) + "/cpulist", &dummy)) break;
+    ++count;
+  }
+  if (n_nodes) *n_nodes = count;
+  if (cpulist && cpulist_cap) {
+    cpulist[0] = 0;
+    if (v >= 0) {
+      if (!read_line(root + "/devices/system/node/node" + std::to_string(v) + "/cpulist", &line))
+        return BSR_ERR_MISSING;
+      cpu_set_t tmp;
+      if (parse_cpulist(line.c_str(), &tmp) < 0) return BSR_ERR_INVALID;
+      if (line.size() + 1 > cpulist_cap) return BSR_ERR_INVALID;
+      memcpy(cpulist, line.c_str(), line.size() + 1);
+    }
+  }
+  return BSR_OK;
+}
+
 int bsr_restore_async(bsr_ctx *c, bsr_req *q, void *cuda_stream) {
   if (!c || !q || q->ctx != c) return BSR_ERR_INVALID;
   std::lock_guard<std::mutex> al(q->async_mu);
@@ -1572,8 +1887,8 @@ int bsr_req_invalid_blocks(bsr_ctx *c, bsr_req *q, uint32_t rank, uint32_t group
 int bsr_req_bitmap(bsr_ctx *c, bsr_req *q, uint64_t *out, size_t words) {
   if (!c || !q || q->ctx != c || (!out && words)) return BSR_ERR_INVALID;
   join_async(q);  // a restore started asynchronously
-  if (words < q->bitmap.size()) return fail(c, BSR_ERR_INVALID, "bitmap buffer too small");
   std::lock_guard<std::mutex> ql(q->mu);
+  if (words < q->bitmap.size()) return fail(c, BSR_ERR_INVALID, "bitmap buffer too small");
   if (!q->bitmap.empty()) memcpy(out, q->bitmap.data(), q->bitmap.size() * 8);
   return BSR_OK;
 }
@@ -1581,9 +1896,9 @@ int bsr_req_bitmap(bsr_ctx *c, bsr_req *q, uint64_t *out, size_t words) {
 int bsr_req_checksums(bsr_ctx *c, bsr_req *q, uint64_t *out, size_t count) {
   if (!c || !q || q->ctx != c || (!out && count)) return BSR_ERR_INVALID;
   join_async(q);  // a restore started asynchronously
+  std::lock_guard<std::mutex> ql(q->mu);
   const size_t cells = (size_t)c->cfg.n_ranks * c->G * q->n_adv;
   if (count < cells) return fail(c, BSR_ERR_INVALID, "checksum buffer too small");
-  std::lock_guard<std::mutex> ql(q->mu);
   if (cells) memcpy(out, q->h_ck, cells * 8);
   return BSR_OK;
 }
@@ -1613,6 +1928,7 @@ int bsr_reset_stats(bsr_ctx *c) {
   c->st = bsr_stats{};
   c->st.slot_bytes = keep.slot_bytes;
   c->st.dev_aux_bytes = keep.dev_aux_bytes;
+  c->st.fill_numa_node = keep.fill_numa_node;
   for (uint32_t r = 0; r < BSR_MAX_RANKS; ++r)
     c->st.ring_bytes_allocated[r] = keep.ring_bytes_allocated[r];
   return BSR_OK;

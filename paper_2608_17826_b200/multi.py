@@ -34,3 +34,25 @@ def max_over_ranks(value: float, device=None, group=None) -> float:
         dist.all_reduce(t, op=dist.ReduceOp.MAX, group=group)
         return float(t.item())
     return float(value)
+
+
+def cpu_share(allowed: list[int], node_cpus_of_rank: list[list[int] | None], local_rank: int) -> list[int]:
+    """The host CPUs local rank `local_rank` keeps for its fill threads when several processes
+    feed their GPUs from one host.
+
+    allowed: CPUs this job may use (its affinity mask).  node_cpus_of_rank[l]: the CPUs of the NUMA
+    node GPU l hangs off, or None where the platform does not say.  Ranks whose GPUs share a node
+    split that node's allowed CPUs evenly, in rank order; ranks without a known node split what no
+    known node claims (all allowed CPUs when no node is known at all).  Every rank gets at least one CPU."""
+    allowed = sorted(allowed)
+    key = [None if c is None else tuple(sorted(set(c) & set(allowed))) or None for c in node_cpus_of_rank]
+    mine = key[local_rank]
+    if mine is None:
+        claimed = set().union(*[set(k) for k in key if k is not None]) if any(k is not None for k in key) else set()
+        pool = [c for c in allowed if c not in claimed] or allowed
+    else:
+        pool = list(mine)
+    peers = [l for l, k in enumerate(key) if k == mine]
+    n, at = len(peers), peers.index(local_rank)
+    lo, hi = at * len(pool) // n, (at + 1) * len(pool) // n
+    return pool[lo:hi] or [pool[min(lo, len(pool) - 1)]]

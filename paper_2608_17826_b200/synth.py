@@ -91,6 +91,14 @@ def mtp_on_layout(seed: int = MASTER_SEED) -> Layout:
     return hetero_layout(seed=seed + 1, bytes_per_token=64976, name="mtp-on-3group-170tensor")
 
 
+def short_run_layout() -> Layout:
+    """A registration dominated by the shortest destination runs a paged cache can have: 1,600
+    tensors of 16 B per token in 16-token blocks (256-byte runs, 80 % of the bytes) beside 50
+    tensors of 128 B per token in 64-token blocks (8 KiB runs).  32,000 B/token, 8,192,000 B per
+    chunk, 25,800 runs per chunk: the stress case for an install kernel's per-run overhead."""
+    return Layout("short-runs-2group-1650tensor", [16, 64], [(0, 16)] * 1600 + [(1, 128)] * 50)
+
+
 def tiny_layout() -> Layout:
     """A very small geometry for brute-force tests: 2 groups, 3 tensors, 16 and 64-token blocks."""
     return Layout("tiny", [16, 64], [(0, 48), (0, 16), (1, 32)])

@@ -1,6 +1,9 @@
 """Builds the same seeded case for the oracle and for the CUDA library, and compares them."""
 from __future__ import annotations
 
+import os
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 
 from oracle import bsr_oracle as O
@@ -22,13 +25,21 @@ class Case:
         self.keys = O.prefix_keys(O.chunk_digests(self.tok, self.salt), self.salt, reg_id)
         self.payload: dict[tuple[int, int], np.ndarray] = {}
         self.cks: dict[tuple[int, int], list[int]] = {}
-        for r in range(R):
-            for i in range(N):
-                if present is not None and not present(r, i):
-                    continue
-                p = synth.chunk_payload(layout, r, i, seed=seed).copy()
-                self.payload[(r, i)] = p
-                self.cks[(r, i)] = O.group_checksums(self.reg, p)
+        todo = [(r, i) for r in range(R) for i in range(N) if present is None or present(r, i)]
+
+        def make(ri):
+            p = synth.chunk_payload(layout, ri[0], ri[1], seed=seed).copy()
+            return ri, p, O.group_checksums(self.reg, p)
+
+        if len(todo) * layout.chunk_bytes > (1 << 30):
+            # a long prefix: draw the chunks (and stamp their stored checksums) on several threads
+            with ThreadPoolExecutor(min(16, os.cpu_count() or 4)) as ex:
+                made = list(ex.map(make, todo))
+        else:
+            made = [make(ri) for ri in todo]
+        for ri, p, ck in made:
+            self.payload[ri] = p
+            self.cks[ri] = ck
         self.pools = [synth.pool_blocks(layout, g, N) for g in range(self.G)]
         self.tables = [[synth.block_table(layout, r, g, N, seed=seed) for g in range(self.G)]
                        for r in range(R)]
@@ -141,6 +152,17 @@ def assert_paged_equal(gpu: GpuSide, oracle_paged):
             if not np.array_equal(got, oracle_paged[r][l]):
                 bad = np.argwhere(got != oracle_paged[r][l])
                 raise AssertionError(f"paged mismatch rank {r} tensor {l}: {len(bad)} bytes, first at {bad[0]}")
+
+
+def assert_paged_equal_on_device(gpu: GpuSide, oracle_paged_dev):
+    """The same comparison, every byte of every paged tensor, against a copy of the oracle's image
+    that already sits in device memory (long prefixes: nothing is downloaded)."""
+    torch, c = gpu.torch, gpu.case
+    for r in range(c.R):
+        for l in range(len(c.layout.tensors)):
+            if not torch.equal(gpu.paged[r][l], oracle_paged_dev[r][l]):
+                bad = (gpu.paged[r][l] != oracle_paged_dev[r][l]).nonzero()
+                raise AssertionError(f"paged mismatch rank {r} tensor {l}: {len(bad)} bytes, first at {bad[0].tolist()}")
 
 
 def run_oracle(case: Case, W: int, n_adv: int | None = None, tiers=None, fetch_fault=None):

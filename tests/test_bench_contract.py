@@ -10,12 +10,16 @@ import pytest
 from conftest import ROOT
 
 
-def test_reference_arm_prints_one_json_line_with_the_contract_keys():
-    env = dict(os.environ, RANK="0", WORLD_SIZE="1")
-    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference",
-                          "--steps", "1", "--warmup", "3"], capture_output=True, text=True, env=env, timeout=600)
+def _reference(extra, env=None, timeout=900):
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--chunks", "4",
+                          "--steps", "1", "--warmup", "3", *extra], capture_output=True, text=True,
+                         env=dict(os.environ, **(env or {})), timeout=timeout)
     assert out.returncode == 0, out.stderr[-2000:]
-    lines = [l for l in out.stdout.splitlines() if l.strip()]
+    return [l for l in out.stdout.splitlines() if l.strip()]
+
+
+def test_reference_arm_prints_one_json_line_with_the_contract_keys():
+    lines = _reference([], env={"RANK": "0", "WORLD_SIZE": "1"})
     assert len(lines) == 1
     d = json.loads(lines[0])
     assert d["impl"] == "reference" and d["higher_is_better"] is True and d["vs_baseline"] is None
@@ -28,18 +32,34 @@ def test_reference_arm_prints_one_json_line_with_the_contract_keys():
     assert d["e2e"]["value"] == d["value"]
 
 
+def test_reference_arm_started_for_two_gpus_without_a_launcher_still_prints_one_line():
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
+                          "--chunks", "4", "--steps", "1", "--warmup", "3"], capture_output=True, text=True,
+                         env=env, timeout=900)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.strip()]
+    assert len(lines) == 1 and json.loads(lines[0])["n_gpus"] == 2
+
+
 def test_other_ranks_of_the_reference_arm_do_no_work():
-    env = dict(os.environ, RANK="1", WORLD_SIZE="2")
-    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference",
-                          "--steps", "1", "--warmup", "3"], capture_output=True, text=True, env=env, timeout=120)
-    assert out.returncode == 0 and out.stdout.strip() == ""
+    assert _reference(["--gpus", "2"], env={"RANK": "1", "WORLD_SIZE": "2"}, timeout=120) == []
+
+
+def test_both_arms_name_the_same_configuration():
+    """The reference arm and the GPU arm describe their workload with the same `config` object."""
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench._config(128) == bench._config(128, "baseline")
+    assert bench._config(128)["workload"] == bench.WORKLOAD["name"]
+    assert bench._config(32)["workload"].startswith("REDUCED to 32 chunks")
 
 
 @pytest.mark.gpu
 def test_gpu_arm_prints_one_json_line_with_every_contract_key():
     """The GPU arm on a reduced prefix (32 chunks; the label says so): one JSON line carrying the
-    metric, the end-to-end figure with its copied bytes, launches, clocks, the roofline of the
-    install kernel and the CPU oracle baseline."""
+    metric, the end-to-end figure with its copied bytes and what bounds it, launches, clocks, the
+    roofline of the install kernel as launched inside the timed steps, and the CPU oracle baseline."""
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--chunks", "32", "--steps", "3",
                           "--warmup", "3"], capture_output=True, text=True, timeout=900)
     assert out.returncode == 0, out.stderr[-2000:]
@@ -48,19 +68,31 @@ def test_gpu_arm_prints_one_json_line_with_every_contract_key():
     d = json.loads(lines[0])
     for k in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better",
               "scaling", "vs_baseline", "dtype", "data", "config", "e2e", "gpu_launches", "clocks", "roofline",
-              "cpu_baseline"):
+              "cpu_baseline", "resident"):
         assert k in d, k
     assert d["n_gpus"] == 1 and d["steps"] == 3 and d["warmup"] >= 3 and d["scaling"] == "weak"
     assert d["value"] > 0 and d["vs_baseline"] is None and d["data"] == "synthetic"
     assert d["config"]["workload"].startswith("REDUCED to 32 chunks")
+    payload = 32 * 2 * 16_408_576
+    # `value` is a restore from the host tier: it cannot beat the link it crosses
     e = d["e2e"]
-    assert 0 < e["value"] < d["value"] and e["unit"] == d["unit"]
-    assert e["h2d_bytes_per_step"] >= 32 * 2 * 16_408_576 and e["d2h_bytes_per_step"] > 0
-    assert d["gpu_launches"] == 2 * 3                       # one probe and one install launch per step
+    assert d["value"] < 1.05 * e["h2d_link_GBps_measured"] and abs(d["value"] - payload / d["ms_per_step"] / 1e6) < 1e-6
+    assert 0.6 * d["value"] < e["value"] < 1.4 * d["value"] and e["unit"] == d["unit"]   # the same path, timed apart
+    assert e["h2d_bytes_per_step"] >= payload + 32 * 256 * 4 and e["d2h_bytes_per_step"] > 0
+    assert e["bound_GBps"] == min(e["h2d_link_GBps_measured"], e["host_fill_only_GBps"], e["host_fill_plus_h2d_GBps"])
+    assert abs(e["frac_of_bound"] - e["value"] / e["bound_GBps"]) < 1e-9
+    # launches: one probe per step plus the install launches, 16 descriptors each on this workload
+    inst = e["install"]
+    assert inst["descriptors_per_launch"] == 16 and inst["launches_per_step"] == 4
+    assert d["gpu_launches"] == 3 * (1 + 4)
     assert set(("sm_mhz", "sm_max_mhz", "reasons")) <= set(d["clocks"])
     r = d["roofline"]
     assert r["bound"] == "hbm" and r["unit"] == "GB/s" and r["kernel"] == "bsr_install_bulk_kernel"
-    assert abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9 and 0.5 < r["frac"] < 1.2
-    assert 0.9 < r["traffic"] / (2 * 32 * 2 * 16_408_576) < 1.1     # measured DRAM bytes ~ algorithmic bytes
+    assert r["launches"] == 3 * 4 and r["algorithmic_bytes_per_launch"] == 2 * 16 * 16_408_576
+    assert abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9 and 0.2 < r["frac"] < 1.2
+    assert abs(r["achieved"] - r["algorithmic_bytes_per_launch"] / r["avg_launch_ms"] / 1e6) < 1e-6
+    res = d["resident"]
+    assert res["descriptors_per_launch"] == 64 and 0.3 < res["frac"] < 1.2
     c = d["cpu_baseline"]
     assert c["kind"] == "oracle" and c["cores"] == 1 and c["value"] > 0 and c["sample"]
+    assert c["all_cores"]["cores"] >= 1 and c["all_cores"]["value"] > 0

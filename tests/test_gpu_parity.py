@@ -341,9 +341,11 @@ def test_direct_install_from_pinned_slots_matches_oracle(layout_name, R, N, W):
 # ---------------------------------------------------------------- kernel choice by registration
 def test_install_kernel_in_use_reports_the_choice():
     from paper_2608_17826_b200 import binding as B
-    want = {"baseline": B.BSR_INSTALL_BULK, "hetero": B.BSR_INSTALL_BULK, "tiny": B.BSR_INSTALL_BULK}
+    # most bytes in runs of at most 1 KiB (moved as spans of several runs): the vector kernel
+    want = {"baseline": B.BSR_INSTALL_BULK, "hetero": B.BSR_INSTALL_BULK, "tiny": B.BSR_INSTALL_VECTOR,
+            "short_runs": B.BSR_INSTALL_VECTOR}
     for name, layout in (("baseline", synth.baseline_layout()), ("hetero", synth.hetero_layout()),
-                         ("tiny", synth.tiny_layout())):
+                         ("tiny", synth.tiny_layout()), ("short_runs", synth.short_run_layout())):
         case = Case(layout, 1, 1, seed=1600)
         with GpuSide(case, 1) as gpu:
             assert B.bsr_install_kernel_in_use(gpu.ctx) == (B.BSR_OK, want[name])
@@ -376,6 +378,110 @@ def test_many_pipeline_shapes_give_the_same_bytes():
                 gpu.B.bsr_reset_stats(gpu.ctx)
                 assert gpu.restore() == gpu.B.BSR_OK, (trial, cfg, gpu.B.bsr_last_error(gpu.ctx))
                 _check_success(case, W, gpu, ora, N)
+
+
+# ---------------------------------------------------------------- install launches take several chunks
+@pytest.mark.parametrize("W,batch,depth,per_launch", [
+    (32, 0, 0, 16),     # defaults: 16 descriptors = 8 chunks of each of the 2 rank slices
+    (16, 0, 0, 8),      # ... but never more than a quarter of the window per rank
+    (16, 4, 0, 4),
+    (16, 64, 3, 6),     # never more chunks per rank than staging buffers
+    (4, 0, 0, 2),
+    (16, 1, 0, 2),      # never less than one chunk of every rank slice
+])
+def test_install_launches_carry_the_configured_number_of_chunks(W, batch, depth, per_launch):
+    layout = synth.Layout("mid", [64, 16], [(0, 1024), (0, 48), (1, 256)])
+    R, N = 2, 48
+    case = Case(layout, R, N, seed=1700)
+    ora = run_oracle(case, W)
+    with GpuSide(case, W, install_batch=batch, dev_staging_depth=depth) as gpu:
+        rc, keys, bm, n_hit = gpu.probe()
+        gpu.request(keys, n_hit)
+        gpu.B.bsr_reset_stats(gpu.ctx)
+        assert gpu.restore() == gpu.B.BSR_OK, gpu.B.bsr_last_error(gpu.ctx)
+        _check_success(case, W, gpu, ora, N)
+        st = gpu.stats()
+        assert st.install_descriptors == R * N
+        assert st.install_launches == -(-R * N // per_launch)
+
+
+def test_a_launch_group_that_cannot_grow_is_not_waited_for():
+    """Two restores share a pool of 2 slots per rank while each would like 4 chunks per launch: neither
+    can ever hold a full group, so a group is launched as soon as nothing else can make progress."""
+    import threading
+    layout = synth.Layout("mid", [64, 16], [(0, 1024), (1, 256)])
+    R, N, W = 2, 12, 16
+    case = Case(layout, R, N, seed=1701)
+    ora = run_oracle(case, W)
+    with GpuSide(case, W, budget_slots=2, timeout_ms=20000) as gpu:
+        B = gpu.B
+        rc, keys, bm, n_hit = gpu.probe()
+        reqs = []
+        for k in range(2):
+            flat = [t for tr in case.tables_prefix(N) for t in tr]
+            rc, q = B.bsr_req_create(gpu.ctx, keys[:N], flat)
+            assert rc == B.BSR_OK
+            reqs.append(q)
+        rcs = [None, None]
+
+        def go(k):
+            rcs[k] = B.bsr_restore(gpu.ctx, reqs[k], None)
+
+        ts = [threading.Thread(target=go, args=(k,)) for k in range(2)]
+        [t.start() for t in ts]
+        [t.join() for t in ts]
+        assert rcs == [B.BSR_OK, B.BSR_OK], B.bsr_last_error(gpu.ctx)
+        for q in reqs:
+            assert B.bsr_commit(gpu.ctx, q) == (B.BSR_OK, N)
+        assert_paged_equal(gpu, ora["paged"])                    # both wrote the same bytes to the same blocks
+        assert gpu.stats().peak_staging_bytes[0] == 2 * case.reg.slot_bytes
+        for q in reqs:
+            B.bsr_req_release(gpu.ctx, q)
+
+
+# ---------------------------------------------------------------- calibration passes install nothing
+def test_calibration_passes_move_the_bytes_but_install_nothing():
+    layout = synth.Layout("mid", [64, 16], [(0, 1024), (0, 48), (1, 256)])
+    R, N, W = 2, 20, 8
+    case = Case(layout, R, N, seed=1702)
+    ora = run_oracle(case, W)
+    with GpuSide(case, W) as gpu:
+        B = gpu.B
+        rc, keys, bm, n_hit = gpu.probe()
+        gpu.request(keys, n_hit)
+        for stages in (B.BSR_CAL_FILL, B.BSR_CAL_FILL_H2D):
+            B.bsr_reset_stats(gpu.ctx)
+            rc, sec = B.bsr_restore_calibrate(gpu.ctx, gpu.req, stages)
+            assert rc == B.BSR_OK and sec > 0
+            st = gpu.stats()
+            assert st.install_launches == 0 and st.bytes_installed[0] == 0
+            assert st.peak_staging_bytes[0] == W * case.reg.slot_bytes       # the same slots were live
+            assert gpu.commit() == 0 and (gpu.bitmap(N) == 0).all()          # nothing was installed ...
+            for r in range(R):
+                for l in range(len(layout.tensors)):
+                    assert bool((gpu.paged[r][l] == synth.CANARY).all())     # ... and no paged byte written
+        assert B.bsr_restore_calibrate(gpu.ctx, gpu.req, 7)[0] == B.BSR_ERR_INVALID
+        # a missing chunk fails a calibration pass like it fails a restore
+        assert B.bsr_tier_remove(gpu.ctx, 1, keys[5]) == B.BSR_OK
+        assert B.bsr_restore_calibrate(gpu.ctx, gpu.req, B.BSR_CAL_FILL)[0] == B.BSR_ERR_MISSING
+        p = case.payload[(1, 5)]
+        assert B.bsr_tier_put(gpu.ctx, 1, keys[5], p, p.size, case.cks[(1, 5)]) == B.BSR_OK
+        # the request is untouched: a real restore afterwards succeeds
+        B.bsr_reset_stats(gpu.ctx)
+        assert gpu.restore() == B.BSR_OK, B.bsr_last_error(gpu.ctx)
+        _check_success(case, W, gpu, ora, N)
+
+
+def test_registration_with_an_empty_group_is_rejected():
+    from paper_2608_17826_b200 import binding as B
+    import torch
+    rc, ctx = B.bsr_ctx_create(2, 1)
+    assert rc == B.BSR_OK
+    t = torch.zeros(64 * 16 * 4, dtype=torch.uint8, device="cuda")
+    assert B.bsr_register(ctx, 0, [(64, 4), (64, 4), (64, 4)], [(0, 16, t.data_ptr()), (2, 16, t.data_ptr())]) \
+        == B.BSR_ERR_INVALID
+    assert "group 1 has no tensor" in B.bsr_last_error(ctx)
+    B.bsr_ctx_destroy(ctx)
 
 
 # ---------------------------------------------------------------- the timeline shows Eq. 3
@@ -471,6 +577,42 @@ def test_more_tiles_per_chunk_than_ctas_in_the_grid(variant, location):
         gpu.request(keys, n_hit)
         assert gpu.restore() == gpu.B.BSR_OK, gpu.B.bsr_last_error(gpu.ctx)
         _check_success(case, W, gpu, ora, N)
+
+
+@pytest.mark.parametrize("variant,location", [(1, 0), (1, 1), (2, 0), (2, 1)])
+@pytest.mark.parametrize("layout_name", ["odd_spans", "short_runs"])
+def test_spans_of_several_short_runs_land_in_their_own_blocks(layout_name, variant, location):
+    """Short destination runs travel in spans of several whole runs whose stores are scattered run by
+    run.  `odd_spans`: 768-byte runs, 21 to a span, 16 to a tensor, so that spans begin in the middle
+    of a tensor and run on into the next one (and the next family, of 256-byte runs, starts at an odd
+    place); `short_runs`: the registration dominated by 256-byte runs, 64 to a span over 4 tensors."""
+    layout = {"odd_spans": synth.Layout("odd_spans", [16, 64], [(0, 48)] * 5 + [(0, 16)] * 7 + [(1, 128)] * 3),
+              "short_runs": synth.short_run_layout()}[layout_name]
+    R, N, W = 2, 5, 2
+    case = Case(layout, R, N, seed=1800 + variant)
+    ora = run_oracle(case, W)
+    with GpuSide(case, W, location=location, install_variant=variant) as gpu:
+        rc, keys, bm, n_hit = gpu.probe()
+        gpu.request(keys, n_hit)
+        assert gpu.restore() == gpu.B.BSR_OK, gpu.B.bsr_last_error(gpu.ctx)
+        _check_success(case, W, gpu, ora, N)
+
+
+def test_stores_of_long_runs_followed_by_a_long_stretch_of_short_run_spans_in_one_cta():
+    """297 spans per chunk (16 pieces of long runs, then 281 spans of 256-byte runs) against a grid of
+    2 x 148 CTAs: CTA b takes span (b - n) mod 297 of chunk n, so the CTAs with small b first issue a
+    few bulk stores and then only spans whose stores are scattered by the sum warps.  The stages of
+    those last bulk stores must be handed back although no further store follows them."""
+    layout = synth.Layout("stores_then_spans", [64, 16], [(0, 512)] * 2 + [(1, 16)] * 1124)
+    R, N, W = 1, 24, 32
+    case = Case(layout, R, N, seed=1900)
+    ora = run_oracle(case, W)
+    for location in (1, 0):
+        with GpuSide(case, W, location=location, install_variant=2, timeout_ms=10000) as gpu:
+            rc, keys, bm, n_hit = gpu.probe()
+            gpu.request(keys, n_hit)
+            assert gpu.restore() == gpu.B.BSR_OK, gpu.B.bsr_last_error(gpu.ctx)
+            _check_success(case, W, gpu, ora, N)
 
 
 def test_admission_stops_at_the_first_failure():

@@ -87,3 +87,26 @@ def test_single_process_needs_no_process_group():
     assert multi.commit_across_ranks(5, 5) == 5
     assert multi.commit_across_ranks(0, 5) == 0
     assert multi.max_over_ranks(3.5) == 3.5
+
+
+def test_cpu_share_splits_each_numa_node_among_the_ranks_whose_gpu_hangs_off_it():
+    """Eight processes on a two-socket host: every rank keeps a quarter of its GPU's node and no CPU
+    is handed out twice; without node information the allowed CPUs are split evenly."""
+    n0 = list(range(0, 16)) + list(range(32, 48))
+    n1 = list(range(16, 32)) + list(range(48, 64))
+    shares = [multi.cpu_share(list(range(64)), [n0] * 4 + [n1] * 4, l) for l in range(8)]
+    assert all(len(s) == 8 for s in shares)
+    assert sorted(c for s in shares for c in s) == list(range(64))
+    assert all(set(s) <= set(n0) for s in shares[:4]) and all(set(s) <= set(n1) for s in shares[4:])
+    # an affinity mask narrower than the node is respected
+    assert multi.cpu_share(list(range(8)), [n0, n0], 1) == [4, 5, 6, 7]
+    # no node known: an even split; more ranks than CPUs: everyone still gets one
+    assert [multi.cpu_share(list(range(16)), [None] * 2, l) for l in range(2)] == [list(range(8)), list(range(8, 16))]
+    assert [multi.cpu_share([0, 1], [None] * 4, l) for l in range(4)] == [[0], [0], [1], [1]]
+
+
+def test_slices_of_a_job_are_dealt_round_robin_and_cover_the_job():
+    for world in (1, 2, 4, 8):
+        got = [multi.slices_of(p, world, 2 * world) for p in range(world)]
+        assert sorted(r for s in got for r in s) == list(range(2 * world))
+        assert all(s == [p, p + world] for p, s in enumerate(got))

@@ -52,13 +52,13 @@ def test_mix64_vector_form_equals_scalar_form():
     assert [int(v) for v in O._mix64_vec(x)] == [O.mix64(int(v)) for v in x]
 
 
-def _survey_tokens(n):
+def _spec_tokens(n):
     return np.array([O.mix64(0xB5A ^ ((j * PHI) & M)) % 129280 for j in range(n)], dtype=np.int32)
 
 
 def test_digest_and_key_golden_vectors():
     g = read_golden("spec_vectors.txt")
-    tok = _survey_tokens(4096)
+    tok = _spec_tokens(4096)
     assert [int(t) for t in tok[:8]] == [int(v) for v in g["tok_first8"]]
     d = O.chunk_digests(tok, salt=7)
     k = O.prefix_keys(d, salt=7, reg_id=1)
@@ -283,6 +283,30 @@ def test_restore_equals_bytewise_definition_on_tiny_input():
             for l, (gg, _) in enumerate(layout.tensors):
                 if gg == g:
                     assert (paged[r][l][spare] == synth.CANARY).all()
+
+
+def test_parallel_for_over_a_window_equals_the_bytewise_definition_and_fails_alike():
+    """The all-cores timing form of the oracle (a thread pool over the chunks of a window) against
+    the same one-byte-at-a-time definition, and its failure report against the serial loop's."""
+    layout = synth.tiny_layout()
+    R, N, W = 2, 7, 3
+    reg, tok, tiers, keys, tables, paged, payload, pools = _build_case(layout, R, N, seed=33)
+    req = O.Request(keys[:N], tables, R, reg.n_groups)
+    status, st_par = O.restore(reg, tiers, req, paged, W, workers=4)
+    assert status == O.OK and req.valid.all() and O.commit(reg, req, paged) == N
+    assert st_par.windows == 3 and st_par.peak_staging_bytes == [W * reg.slot_bytes] * R
+    assert st_par.bytes_installed == [N * reg.chunk_bytes] * R
+    want = _brute_force_paged(layout, R, N, tables, payload, pools)
+    for r in range(R):
+        for l in range(len(layout.tensors)):
+            assert np.array_equal(paged[r][l], want[r][l])
+    # a corrupted word in the second window: same status, nothing valid, nothing exposed
+    bad = payload[(1, 4)]
+    bad[8] ^= 0x40
+    for workers in (1, 4):
+        req = O.Request(keys[:N], tables, R, reg.n_groups)
+        status, _ = O.restore(reg, tiers, req, paged, W, workers=workers)
+        assert status == O.ERR_CHECKSUM and not req.valid.any() and O.commit(reg, req, paged) == 0
 
 
 @settings(max_examples=25, deadline=None, derandomize=True)
