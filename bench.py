@@ -65,7 +65,7 @@ def _peaks():
     if os.path.exists(p):
         with open(p) as f:
             return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
-    return 6650.0, "fallback (earlier pool measurement)"
+    return 6650.0, "fallback (an earlier measurement of the same copy on a B200)"
 
 
 class ClockSampler:
@@ -301,7 +301,7 @@ def place_on_host(torch, B, local, world):
     for l in range(world):
         cpus = None
         try:
-            p = torch.cuda.get_device_properties(l)
+            p = torch.cuda.get_device_properties(l if l < torch.cuda.device_count() else 0)
             bus = f"{p.pci_domain_id:04x}:{p.pci_bus_id:02x}:{p.pci_device_id:02x}.0"
             rc, node, cpulist, _ = B.bsr_numa_of_pci("/sys", bus)
             if rc == B.BSR_OK and node >= 0 and cpulist:
@@ -309,7 +309,7 @@ def place_on_host(torch, B, local, world):
                 for part in cpulist.split(","):
                     lo, _, hi = part.partition("-")
                     cpus += list(range(int(lo), int(hi or lo) + 1))
-        except (AttributeError, RuntimeError, ValueError):
+        except (AttributeError, AssertionError, RuntimeError, ValueError):
             cpus = None
         node_cpus.append(cpus)
     mine = multi.cpu_share(allowed, node_cpus, local)
@@ -477,8 +477,8 @@ def run_gpu(args):
                  "e2e": ("token ids, block tables and tier in host memory; request created in the step; bitmap "
                          "read back; " + ("install kernel reads the slots over the link" if args.direct else
                                           "host tier -> pinned pool -> H2D -> install")),
-                 "load_concurrency": args.load_concurrency, "dev_staging_depth": args.depth or 12,
-                 "install_batch": args.install_batch or 16, "fill_cpus": len(cpus), "fill_numa_node": numa_node},
+                 "load_concurrency": args.load_concurrency, "dev_staging_depth": args.depth or 20,
+                 "install_batch": args.install_batch or 32, "fill_cpus": len(cpus), "fill_numa_node": numa_node},
         "per_rank_GBps": value / (world * R),
         "restore_seconds": ms_val / 1e3,
         "frac_of_h2d_link": value / world / h2d_gbs,
@@ -576,6 +576,7 @@ def spawn_ranks(args):
     for r in range(args.gpus):
         env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(args.gpus),
                    LOCAL_WORLD_SIZE=str(args.gpus), MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        env.setdefault("NCCL_DEBUG", "INFO")  # the communicator's own log (ranks, transport) goes to stderr
         procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__), *sys.argv[1:]], env=env,
                                       stdout=None if r == 0 else subprocess.DEVNULL))
     worst = 0

@@ -74,7 +74,7 @@ typedef struct bsr_config {
   uint32_t load_concurrency;  /* threads copying tier objects into staging slots (Table 1 "FS
                                  load concurrency": changes throughput, never W or the peak)     */
   uint32_t dev_staging_depth; /* D >= 1 device staging buffers per rank (bounded auxiliary state,
-                                 M_aux of Eq. 4; independent of the prefix length); 0 = 12       */
+                                 M_aux of Eq. 4; independent of the prefix length); 0 = 20       */
   uint32_t timeout_ms;        /* deadline of one bsr_restore call; 0 = 30,000                    */
   uint32_t slot_align;        /* staging slot size = chunk bytes rounded up to this; 0 = 4096    */
   int32_t device;             /* CUDA device ordinal                                             */
@@ -92,9 +92,9 @@ typedef struct bsr_config {
                                  run concurrently and share a pool of B slots per rank; each holds
                                  at most W, together never more than B                            */
   uint32_t install_batch;     /* chunk descriptors (chunk x rank) one install launch takes on the
-                                 path through the slot pool; 0 = 16.  A launch waits until that many
+                                 path through the slot pool; 0 = 32.  A launch waits until that many
                                  chunks have been queued for copying: never more per rank than D or
-                                 W / 4, never fewer than one chunk of every rank, and never while
+                                 W / 2, never fewer than one chunk of every rank, and never while
                                  nothing else could make progress.  Larger launches run the kernel
                                  nearer device-copy speed, smaller ones hand slots back sooner.
                                  Changes throughput only, never W or the peak                      */

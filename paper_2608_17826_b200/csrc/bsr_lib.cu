@@ -835,13 +835,15 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
   const bool direct = c->cfg.direct_install != 0 && stages == kStagesAll;
   const uint32_t n_ev = res->n_slots;  // launch slots: a scratch set and three events each
   // Chunks of each rank that one install launch takes.  A launch costs about 13 us on top of its
-  // bytes (25 us while the copy engine is busy, which here it always is), so a single 16 MB chunk
-  // (5 us of traffic) runs at a fraction of device-copy speed and 16 chunks at three quarters of
-  // it; fewer chunks per launch hand the window's slots back sooner.  A launch never needs more
-  // staging buffers than a rank has, and leaves three quarters of the window to the fill.
+  // bytes (read-only ramp, write-only tail, address look-ups, the last CTA's verdicts), so a single
+  // 16 MB chunk (5 us of traffic) runs at a third of device-copy speed, 16 chunks at 0.72 and 32 at
+  // 0.88.  A launch never needs more staging buffers than a rank has, and leaves half of the window
+  // to the fill: measured on B200, restore throughput is the same with half the window waiting for
+  // its launch as with one chunk per launch (the fill threads only need a few free slots ahead),
+  // and the peak stays W slots either way.
   uint32_t cpl = c->cfg.install_batch / R;
   if (cpl > D) cpl = D;
-  if (cpl > W / 4) cpl = W / 4;
+  if (cpl > W / 2) cpl = W / 2;
   if (cpl > BSR_K_MAX_BATCH / R) cpl = BSR_K_MAX_BATCH / R;
   if (cpl == 0) cpl = 1;
   // items (chunk, rank) per launch; a kernel that reads pinned slots over the link takes one
@@ -1254,8 +1256,8 @@ int bsr_ctx_create(const bsr_config *cfg, bsr_ctx **out) {
     c->cfg.load_concurrency = hw < 4 ? 4 : (hw > 16 ? 16 : hw);
   }
   if (c->cfg.load_concurrency > 64) c->cfg.load_concurrency = 64;
-  if (c->cfg.dev_staging_depth == 0) c->cfg.dev_staging_depth = 12;
-  if (c->cfg.install_batch == 0) c->cfg.install_batch = 16;
+  if (c->cfg.dev_staging_depth == 0) c->cfg.dev_staging_depth = 20;
+  if (c->cfg.install_batch == 0) c->cfg.install_batch = 32;
   if (c->cfg.dev_staging_depth > 16) c->cfg.dev_staging_depth = 16;
   if (c->cfg.timeout_ms == 0) c->cfg.timeout_ms = 30000;
   if (c->cfg.slot_align == 0) c->cfg.slot_align = 4096;

@@ -382,11 +382,11 @@ def test_many_pipeline_shapes_give_the_same_bytes():
 
 # ---------------------------------------------------------------- install launches take several chunks
 @pytest.mark.parametrize("W,batch,depth,per_launch", [
-    (32, 0, 0, 16),     # defaults: 16 descriptors = 8 chunks of each of the 2 rank slices
-    (16, 0, 0, 8),      # ... but never more than a quarter of the window per rank
+    (32, 0, 0, 32),     # defaults: 32 descriptors = 16 chunks of each of the 2 rank slices
+    (16, 0, 0, 16),     # ... but never more than half of the window per rank
     (16, 4, 0, 4),
     (16, 64, 3, 6),     # never more chunks per rank than staging buffers
-    (4, 0, 0, 2),
+    (4, 0, 0, 4),
     (16, 1, 0, 2),      # never less than one chunk of every rank slice
 ])
 def test_install_launches_carry_the_configured_number_of_chunks(W, batch, depth, per_launch):

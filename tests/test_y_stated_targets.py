@@ -17,7 +17,7 @@ def test_install_kernel_reaches_its_stated_share_of_the_measured_copy_rate():
     """The stated target for the install kernel: at least 70 % of the measured HBM copy rate in read +
     write traffic, both over all 256 chunk descriptors in one launch and as launched, a few chunks
     at a time, inside a restore from the host tier.  The denominator is the figure measured for this
-    machine pool when one is on file; without it the test has nothing to compare with."""
+    machine when one is on file; without it the test has nothing to compare with."""
     peaks = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if not os.path.exists(peaks):
         pytest.skip("no measured peak on file")
@@ -28,8 +28,7 @@ def test_install_kernel_reaches_its_stated_share_of_the_measured_copy_rate():
     assert out.returncode == 0, out.stderr[-2000:]
     d = json.loads([l for l in out.stdout.splitlines() if l.strip()][-1])
     assert d["resident"]["achieved"] >= 0.70 * hbm, d["resident"]
-    # inside a restore a launch carries 16 descriptors and pays a fixed cost while the copy engine is
-    # busy: 0.73-0.76 of the copy rate measured; the floor leaves room for a busy neighbour
-    assert d["roofline"]["descriptors_per_launch"] >= 16 and d["roofline"]["achieved"] >= 0.65 * hbm, d["roofline"]
+    # inside a restore a launch carries 32 descriptors (0.88 of the copy rate measured)
+    assert d["roofline"]["descriptors_per_launch"] >= 32 and d["roofline"]["achieved"] >= 0.70 * hbm, d["roofline"]
     assert d["e2e"]["frac_of_h2d_link"] >= 0.80, d["e2e"]
     assert d["staging_residual_bytes"] == [0, 0]
