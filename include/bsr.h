@@ -175,12 +175,10 @@ const char *bsr_last_error(bsr_ctx *ctx);
 int bsr_register(bsr_ctx *ctx, uint32_t rank, const bsr_group_desc *groups, uint32_t n_groups,
                  const bsr_tensor_desc *tensors, uint32_t n_tensors);
 
-/* Which install kernel the context launches for sources in device memory under the registration:
- * BSR_INSTALL_BULK or BSR_INSTALL_VECTOR.  BSR_INSTALL_AUTO means the bulk-copy kernel unless more
- * than half of a chunk's bytes sit in destination runs of at most 1 KiB (which travel as spans of
- * several runs and are stored with vector stores in either kernel: there the vector kernel is
- * ahead); direct_install always reads host slots with the vector kernel.
- * Errors: STATE (not every rank registered yet), CUDA. */
+/* Which install kernel the context launches for sources in device memory: BSR_INSTALL_BULK or
+ * BSR_INSTALL_VECTOR.  BSR_INSTALL_AUTO means the bulk-copy kernel (level with or ahead of the vector
+ * kernel on every registration measured); direct_install always reads host slots with the vector
+ * kernel.  Errors: STATE (not every rank registered yet), CUDA. */
 int bsr_install_kernel_in_use(bsr_ctx *ctx, int *variant);
 
 /* Bytes of one chunk and of one staging slot under the current registration. */

@@ -161,7 +161,8 @@ struct bsr_ctx {
   uint32_t pieces = 1;  // fill pieces per chunk
   std::atomic<bool> finalized{false};
   bool use_bulk = true;  // the install kernel chosen for this registration (see finalize_registration)
-  bool has_spans = false;  // the tile table holds spans of several runs
+  bool has_spans = false;     // the tile table holds spans of several runs
+  bool mostly_spans = false;  // ... and they carry more than half of a chunk's bytes
   std::vector<BsrTile> h_tiles;
   BsrTile *d_tiles = nullptr;
   uint64_t *d_tensor_base = nullptr;
@@ -328,25 +329,26 @@ int finalize_registration(bsr_ctx *c) {
   CU(c, cudaMemcpy(c->d_tensor_group, tgroup.data(), c->L * 4, cudaMemcpyHostToDevice));
   CU(c, cudaMalloc(&c->d_tensor_run, c->L * 4));
   CU(c, cudaMemcpy(c->d_tensor_run, trun.data(), c->L * 4, cudaMemcpyHostToDevice));
-  CU(c, cudaFuncSetAttribute(bsr_install_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             BSR_K_BULK_SMEM));
+  CU(c, cudaFuncSetAttribute(bsr_install_bulk_kernel<BSR_K_BULK_SUM_WARPS>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, BSR_K_BULK_SMEM));
+  CU(c, cudaFuncSetAttribute(bsr_install_bulk_kernel<BSR_K_BULK_SUM_WARPS_SPANS>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, BSR_K_BULK_SMEM));
   {
     std::lock_guard<std::mutex> g(c->mu);
     c->st.dev_aux_bytes += c->h_tiles.size() * sizeof(BsrTile) + bases.size() * 8 + c->L * 8;
   }
-  // Kernel choice.  Measured on B200, 256-descriptor launches: where most bytes sit in runs that
-  // travel on their own the bulk-copy kernel runs at the speed of a device copy (1.28 ms on the
-  // baseline registration; the vector kernel needs full occupancy to come within 5 % of it).  Where
-  // most bytes sit in short runs, moved as spans of several runs, every store is a 16-byte vector
-  // store in either kernel, and the vector kernel has sixteen times the warps to issue them with
-  // (0.89 against 0.76 of the copy rate on a registration of 256-byte runs).
+  // Kernel choice.  Measured on B200, 256-descriptor launches: the bulk-copy kernel runs at the
+  // speed of a device copy where the bytes sit in runs that travel on their own (1.28 ms on the
+  // baseline registration) and, with eight sum warps to issue the scattered stores of short-run
+  // spans, at 0.91 of it on a registration of 256-byte runs, ahead of the vector kernel on every
+  // registration tried (0.89 there, 0.86 on the 170-tensor one).  So BSR_INSTALL_AUTO means the
+  // bulk-copy kernel; the vector kernel serves direct_install and an explicit request.
   uint64_t span_bytes = 0;
   for (const BsrTile &tl : c->h_tiles)
     if (tl.n_runs > 1) span_bytes += tl.bytes;
   c->has_spans = span_bytes != 0;
-  const bool mostly_short_runs = 2 * span_bytes > c->chunk_bytes;
-  c->use_bulk = c->cfg.install_variant == BSR_INSTALL_BULK ||
-                (c->cfg.install_variant == BSR_INSTALL_AUTO && !mostly_short_runs);
+  c->mostly_spans = 2 * span_bytes > c->chunk_bytes;
+  c->use_bulk = c->cfg.install_variant != BSR_INSTALL_VECTOR;
   c->finalized.store(true, std::memory_order_release);
   return BSR_OK;
 }
@@ -385,8 +387,13 @@ int launch_install(bsr_ctx *c, const BsrInstallParams &p, cudaStream_t s, StatDe
 #ifdef BSR_K_BULK_MAX_GRID  // test builds: few CTAs, so that each one cycles its stage ring many times
     if (want > BSR_K_BULK_MAX_GRID) want = BSR_K_BULK_MAX_GRID;
 #endif
-    bsr_install_bulk_kernel<<<(uint32_t)(total < want ? total : want), BSR_K_BULK_THREADS,
-                              BSR_K_BULK_SMEM, s>>>(p);
+    const uint32_t grid = (uint32_t)(total < want ? total : want);
+    if (c->mostly_spans)
+      bsr_install_bulk_kernel<BSR_K_BULK_SUM_WARPS_SPANS>
+          <<<grid, BSR_K_BULK_THREADS(BSR_K_BULK_SUM_WARPS_SPANS), BSR_K_BULK_SMEM, s>>>(p);
+    else
+      bsr_install_bulk_kernel<BSR_K_BULK_SUM_WARPS>
+          <<<grid, BSR_K_BULK_THREADS(BSR_K_BULK_SUM_WARPS), BSR_K_BULK_SMEM, s>>>(p);
   } else {
     // About nine tiles per CTA, in whole waves of the 8 CTAs an SM holds: many more CTAs than are
     // resident let the hardware scheduler even out the tail (measured best on B200; one tile per

@@ -96,3 +96,22 @@ def test_gpu_arm_prints_one_json_line_with_every_contract_key():
     c = d["cpu_baseline"]
     assert c["kind"] == "oracle" and c["cores"] == 1 and c["value"] > 0 and c["sample"]
     assert c["all_cores"]["cores"] >= 1 and c["all_cores"]["value"] > 0
+
+
+@pytest.mark.gpu
+def test_two_ranks_started_by_the_benchmark_itself_print_one_line():
+    """`--gpus 2` without a launcher: the script starts its two ranks, they rendezvous on the loopback
+    address, exchange the commit word every step, and rank 0 prints the one line with n_gpus = 2.  On a
+    box with one GPU both ranks drive GPU 0 (their kernels never wait on one another) and the word travels
+    over gloo; the line says so and its figures mean nothing."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--dry-run-one-gpu",
+                          "--chunks", "16", "--steps", "3", "--warmup", "3"], capture_output=True, text=True,
+                         env=env, timeout=900)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.strip()]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["n_gpus"] == 2 and d["dry_run_one_gpu"] is True and d["scaling"] == "weak"
+    assert d["value"] > 0 and d["staging_residual_bytes"] == [16 * 16_408_576 - 32 * 16_408_576] * 2   # N < W
+    assert d["cpu_baseline"]["value"] is None                    # the oracle is timed at one GPU only

@@ -341,9 +341,8 @@ def test_direct_install_from_pinned_slots_matches_oracle(layout_name, R, N, W):
 # ---------------------------------------------------------------- kernel choice by registration
 def test_install_kernel_in_use_reports_the_choice():
     from paper_2608_17826_b200 import binding as B
-    # most bytes in runs of at most 1 KiB (moved as spans of several runs): the vector kernel
-    want = {"baseline": B.BSR_INSTALL_BULK, "hetero": B.BSR_INSTALL_BULK, "tiny": B.BSR_INSTALL_VECTOR,
-            "short_runs": B.BSR_INSTALL_VECTOR}
+    want = {"baseline": B.BSR_INSTALL_BULK, "hetero": B.BSR_INSTALL_BULK, "tiny": B.BSR_INSTALL_BULK,
+            "short_runs": B.BSR_INSTALL_BULK}
     for name, layout in (("baseline", synth.baseline_layout()), ("hetero", synth.hetero_layout()),
                          ("tiny", synth.tiny_layout()), ("short_runs", synth.short_run_layout())):
         case = Case(layout, 1, 1, seed=1600)
