@@ -43,8 +43,12 @@ WORKLOAD = dict(name="32768-token prefix, 128 chunks x 16,408,576 B, 2 rank slic
                      "baseline 2-group/99-tensor layout, 64-token blocks",
                 n_chunks=128, n_ranks=2, W=32)
 # dram read + write bytes per payload byte, from one ncu capture of each install kernel on a
-# 64-descriptor launch (traffic grows in proportion to the descriptors a launch carries)
-NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = {"bsr_install_bulk_kernel": 1.957, "bsr_install_vec_kernel": 1.955}
+# 64-descriptor launch (traffic grows in proportion to the descriptors a launch carries); captured
+# on the baseline and on the short-run registration, the others are scaled with the baseline figure
+NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = {("bsr_install_bulk_kernel", "baseline"): 1.955,
+                                   ("bsr_install_vec_kernel", "baseline"): 1.955,
+                                   ("bsr_install_bulk_kernel", "short_runs"): 1.903,
+                                   ("bsr_install_vec_kernel", "short_runs"): 1.946}
 METRIC, UNIT = "restore GB/s from the host tier (all rank slices; per-rank = value / rank slices)", "GB/s"
 LAYOUTS = {"baseline": synth.baseline_layout, "hetero": synth.hetero_layout, "mtp_on": synth.mtp_on_layout,
            "short_runs": synth.short_run_layout}
@@ -443,7 +447,8 @@ def run_gpu(args):
     k_ms = st_val.install_kernel_ms / max(1, k_launches)
     per_launch_payload = chunk * k_desc / max(1, k_launches)
     achieved = 2 * per_launch_payload / (k_ms / 1e3) / 1e9 if k_ms > 0 else None
-    traffic = NCU_DRAM_BYTES_PER_PAYLOAD_BYTE[kernel_name] * per_launch_payload
+    traffic_key = (kernel_name, args.layout if (kernel_name, args.layout) in NCU_DRAM_BYTES_PER_PAYLOAD_BYTE else "baseline")
+    traffic = NCU_DRAM_BYTES_PER_PAYLOAD_BYTE[traffic_key] * per_launch_payload
     bounds = {"h2d link": h2d_gbs, "host fill alone (tier -> slot copies)": cal["fill_only"],
               "host memory system (fill and the copy engine's reads together)": cal["fill_plus_h2d"]}
     bound_name = min(bounds, key=bounds.get)
@@ -504,6 +509,9 @@ def run_gpu(args):
                      "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
                      "frac": (achieved / hbm_peak) if achieved else None,
                      "traffic": traffic, "peak_source": peak_src,
+                     "traffic_source": f"ncu dram bytes per payload byte of a 64-descriptor launch of this kernel "
+                                       f"({traffic_key[1]} registration: {NCU_DRAM_BYTES_PER_PAYLOAD_BYTE[traffic_key]}) "
+                                       f"x the payload of one launch",
                      "launches": k_launches, "avg_launch_ms": k_ms,
                      "descriptors_per_launch": k_desc / max(1, k_launches),
                      "algorithmic_bytes_per_launch": 2 * per_launch_payload},

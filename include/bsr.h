@@ -242,7 +242,9 @@ int bsr_req_release(bsr_ctx *ctx, bsr_req *req);
  * its admission, before the fill, until its install has been observed complete), copied to a
  * device staging buffer on the library's copy stream, then verified and scattered through the
  * block tables by the install kernel on `cuda_stream` (a cudaStream_t, or NULL for a stream owned
- * by the library).  Objects that live in device memory are installed in place.  The first
+ * by the library).  One install launch takes the chunks queued since the previous one (see
+ * bsr_config.install_batch); their slots are released together when the launch has been observed
+ * complete.  Objects that live in device memory are installed in place.  The first
  * missing key, checksum mismatch, transfer error or deadline overrun stops admission, drains what
  * is in flight, invalidates the whole request and is returned.  Blocking; on return no slot is
  * live and every kernel of the call has finished.

@@ -59,6 +59,29 @@ def test_config2_every_paged_byte_both_launch_configurations():
             assert_paged_equal(gpu, ora["paged"])
 
 
+def test_short_run_registration_64_descriptors_per_launch_every_paged_byte():
+    """The registration dominated by 256-byte runs (25,800 runs per chunk) at 32 chunks x 2 rank slices:
+    through the window (32-descriptor launches) and with all 64 descriptors in one launch, both kernels."""
+    layout = synth.short_run_layout()
+    R, N, W = 2, 32, 32
+    case = Case(layout, R, N, seed=6006)
+    ora = run_oracle(case, W)
+    assert ora["status"] == O.OK and ora["exposed"] == N
+    for location, variant in ((0, 0), (1, 0), (1, 1)):
+        with GpuSide(case, W, location=location, install_variant=variant) as gpu:
+            B = gpu.B
+            rc, keys, bm, n_hit = gpu.probe()
+            assert rc == B.BSR_OK and n_hit == N and np.array_equal(keys, ora["keys"])
+            gpu.request(keys, N)
+            assert gpu.restore() == B.BSR_OK, B.bsr_last_error(gpu.ctx)
+            assert gpu.commit() == N
+            assert np.array_equal(gpu.bitmap(N), ora["req"].bitmap())
+            st = gpu.stats()
+            assert st.install_descriptors == R * N and st.install_launches == (2 if location == 0 else 1)
+            assert st.bytes_installed[0] == st.bytes_installed[1] == N * 8_192_000
+            assert_paged_equal(gpu, ora["paged"])
+
+
 # ---------------------------------------------------------------- big cases with a cyclic tier
 _OBJ_CACHE: dict = {}
 

@@ -471,6 +471,28 @@ def test_calibration_passes_move_the_bytes_but_install_nothing():
         _check_success(case, W, gpu, ora, N)
 
 
+def test_fill_threads_bound_to_the_gpus_numa_node_restore_the_same_bytes():
+    """numa_bind = ALWAYS binds the fill threads and the thread that allocates the pinned pool to the CPUs
+    of the GPU's NUMA node whenever the platform names one (on a single-node host that is every CPU the
+    process may use); OFF never binds.  Either way the restore is the same and the stats say what was done."""
+    import os
+    layout = synth.Layout("mid", [64, 16], [(0, 1024), (0, 48), (1, 256)])
+    R, N, W = 2, 20, 8
+    case = Case(layout, R, N, seed=1703)
+    ora = run_oracle(case, W)
+    allowed = sorted(os.sched_getaffinity(0))
+    for mode in ("off", "always"):
+        from paper_2608_17826_b200 import binding as B
+        with GpuSide(case, W, numa_bind=B.BSR_NUMA_OFF if mode == "off" else B.BSR_NUMA_ALWAYS) as gpu:
+            rc, keys, bm, n_hit = gpu.probe()
+            gpu.request(keys, n_hit)
+            assert gpu.restore() == B.BSR_OK, B.bsr_last_error(gpu.ctx)
+            _check_success(case, W, gpu, ora, N)
+            node = gpu.stats().fill_numa_node
+            assert node == -1 if mode == "off" else node >= -1
+    assert sorted(os.sched_getaffinity(0)) == allowed            # the caller's own mask is never touched
+
+
 def test_registration_with_an_empty_group_is_rejected():
     from paper_2608_17826_b200 import binding as B
     import torch
