@@ -384,7 +384,10 @@ def run_gpu(args):
     torch.cuda.empty_cache()
     hbm_peak, peak_src = _peaks()
     res_payload = step_bytes * args.steps / max(1, res_launches)
+    res_span_ms = st_res.install_span_ms / max(1, res_launches)
     resident = {"what": "install kernel alone: tier objects placed in HBM, probe + install + commit, no host link",
+                "in_kernel_span_ms": res_span_ms,
+                "frac_in_kernel": 2 * res_payload / (res_span_ms / 1e3) / 1e9 / hbm_peak if res_span_ms else None,
                 "GBps_payload": step_bytes / (ms_res / 1e3) / 1e9, "ms_per_step": ms_res,
                 "descriptors_per_launch": int(st_res.install_descriptors) / max(1, res_launches),
                 "avg_launch_ms": res_k_ms, "achieved": 2 * res_payload / (res_k_ms / 1e3) / 1e9 if res_k_ms else None,
@@ -445,6 +448,7 @@ def run_gpu(args):
     k_launches = int(st_val.install_launches)
     k_desc = int(st_val.install_descriptors)
     k_ms = st_val.install_kernel_ms / max(1, k_launches)
+    k_span_ms = st_val.install_span_ms / max(1, k_launches)
     per_launch_payload = chunk * k_desc / max(1, k_launches)
     achieved = 2 * per_launch_payload / (k_ms / 1e3) / 1e9 if k_ms > 0 else None
     traffic_key = (kernel_name, args.layout if (kernel_name, args.layout) in NCU_DRAM_BYTES_PER_PAYLOAD_BYTE else "baseline")
@@ -513,6 +517,11 @@ def run_gpu(args):
                                        f"({traffic_key[1]} registration: {NCU_DRAM_BYTES_PER_PAYLOAD_BYTE[traffic_key]}) "
                                        f"x the payload of one launch",
                      "launches": k_launches, "avg_launch_ms": k_ms,
+                     "in_kernel": {"what": "the same launches timed by the kernel itself: first CTA's start to the last "
+                                           "CTA's end (%globaltimer), i.e. without launch and completion latency",
+                                   "avg_span_ms": k_span_ms,
+                                   "achieved": 2 * per_launch_payload / (k_span_ms / 1e3) / 1e9 if k_span_ms else None,
+                                   "frac": 2 * per_launch_payload / (k_span_ms / 1e3) / 1e9 / hbm_peak if k_span_ms else None},
                      "descriptors_per_launch": k_desc / max(1, k_launches),
                      "algorithmic_bytes_per_launch": 2 * per_launch_payload},
         "resident": resident,

@@ -80,8 +80,10 @@ typedef struct bsr_config {
   int32_t device;             /* CUDA device ordinal                                             */
   uint64_t reg_id;            /* registration identity mixed into every prefix key               */
   uint32_t install_variant;   /* BSR_INSTALL_*                                                   */
-  uint32_t time_kernels;      /* nonzero: bracket every install launch with CUDA events and
-                                 accumulate bsr_stats.install_kernel_ms                          */
+  uint32_t time_kernels;      /* nonzero: bracket every install launch with CUDA events and accumulate
+                                 bsr_stats.install_kernel_ms; the kernels also note their own span
+                                 (first CTA's start to the last CTA's end, one atomic per CTA) in
+                                 bsr_stats.install_span_ms                                        */
   uint32_t direct_install;    /* nonzero: no device staging and no copy-engine transfer; the install
                                  kernel reads the pinned slots over the host link itself (the
                                  staging-free design point of the paper's "Avoiding staging"
@@ -140,6 +142,10 @@ typedef struct bsr_stats {
   uint64_t install_descriptors;                 /* chunk descriptors those install launches carried  */
   int64_t fill_numa_node;                       /* node the fill threads and the pool are bound to,
                                                    -1 = not bound (see bsr_config.numa_bind)          */
+  double install_span_ms;                       /* sum of the launches' in-kernel spans (time_kernels):
+                                                   install_kernel_ms minus launch and completion
+                                                   latency; a restore of device-resident objects that
+                                                   needs more than 8 launches adds nothing here       */
 } bsr_stats;
 
 /* ---- context ------------------------------------------------------------------------------- */
@@ -269,7 +275,8 @@ int bsr_restore_wait(bsr_ctx *ctx, bsr_req *req, int *restore_status);
  * they are; byte counters are not advanced (the peak meter is: slots were live).  *seconds = host
  * wall time of the pass.  Comparing request bytes / seconds of the two forms with the link rate
  * and with a full restore tells which stage bounds a restore on this host.
- * Errors: INVALID, and whatever a restore can return for a missing key or a failed copy. */
+ * Errors: INVALID, STATE (BSR_CAL_FILL_H2D on a direct_install context, which has no device staging),
+ * and whatever a restore can return for a missing key or a failed copy. */
 enum { BSR_CAL_FILL = 1, BSR_CAL_FILL_H2D = 2 };
 int bsr_restore_calibrate(bsr_ctx *ctx, bsr_req *req, int stages, double *seconds);
 

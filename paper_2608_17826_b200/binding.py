@@ -76,7 +76,8 @@ class bsr_stats(C.Structure):
                 ("h2d_copies", C.c_uint64), ("install_launches", C.c_uint64),
                 ("bytes_restored_by_tier", C.c_uint64 * 4),
                 ("install_kernel_ms", C.c_double), ("last_restore_ms", C.c_double),
-                ("install_descriptors", C.c_uint64), ("fill_numa_node", C.c_int64)]
+                ("install_descriptors", C.c_uint64), ("fill_numa_node", C.c_int64),
+                ("install_span_ms", C.c_double)]
 
 
 class bsr_trace_rec(C.Structure):

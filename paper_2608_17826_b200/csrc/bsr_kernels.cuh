@@ -86,6 +86,9 @@ struct BsrInstallParams {
   unsigned int *err_flag;    // host-mapped word, set to nonzero if a bounded wait gave up (bulk variant)
   uint64_t *ck_out;          // [(r*G + g) * n_adv + i] computed checksum
   uint32_t *verdict;         // same index: 1 verified, 2 mismatch
+  uint64_t *span_start;      // scratch word (zero on entry, zeroed on exit) and ...
+  uint64_t *span_out;        // ... host-mapped word for the launch's in-kernel span in ns (first CTA's start to
+                             // the last CTA's verdict pass); NULL = not measured
   uint64_t wait_ns;          // bound of every wait inside the bulk kernel; 0 = BSR_K_WAIT_NS
   uint32_t stall_tile;       // test hook: work item whose load is never issued; ~0u = none
   uint32_t pad0;
@@ -105,6 +108,19 @@ __device__ __forceinline__ uint64_t bsr_mix64(uint64_t x) {
   x = (x ^ (x >> 32)) * BSR_K_PHI;
   x = (x ^ (x >> 29)) * BSR_K_PHI;
   return x ^ (x >> 32);
+}
+
+__device__ __forceinline__ uint64_t bsr_globaltimer() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+// In-kernel span of a launch, for measurement runs: every CTA notes its start (the earliest wins),
+// the last CTA to finish publishes now - earliest.  Costs one atomic per CTA when enabled.
+__device__ __forceinline__ void bsr_span_begin(const uint64_t *span_out, uint64_t *span_start) {
+  if (span_out && threadIdx.x == 0)
+    atomicMax((unsigned long long *)span_start, (unsigned long long)~bsr_globaltimer());
 }
 
 __device__ __forceinline__ uint64_t bsr_warp_sum(uint64_t v) {
@@ -179,7 +195,14 @@ __device__ __forceinline__ void bsr_install_finish(const BsrInstallParams &p) {
     p.ck_out[o] = s;
     p.verdict[o] = (s == cd.expect[g]) ? 1u : 2u;
   }
-  if (threadIdx.x == 0) *p.ctas_done = 0u;
+  if (threadIdx.x == 0) {
+    *p.ctas_done = 0u;
+    if (p.span_out) {
+      const uint64_t first = ~__ldcg((const unsigned long long *)p.span_start);
+      *p.span_start = 0ull;
+      *reinterpret_cast<volatile uint64_t *>(p.span_out) = bsr_globaltimer() - first;
+    }
+  }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -191,6 +214,7 @@ template <int THREADS, int UNROLL, bool SPANS>
 __global__ void __launch_bounds__(THREADS, 2048 / THREADS)  // full occupancy: 32 registers at 256 threads
 bsr_install_vec_kernel(const __grid_constant__ BsrInstallParams p) {
   __shared__ uint64_t red[THREADS / 32];
+  bsr_span_begin(p.span_out, p.span_start);
   const uint32_t total = p.n_chunks * p.n_tiles;
   uint64_t sum = 0;
   int cur_c = -1, cur_g = -1;
@@ -321,11 +345,6 @@ static_assert(BSR_K_BULK_STAGES <= 32, "the meta ring assumes the other warps tr
 __device__ __forceinline__ uint32_t bsr_smem_u32(const void *p) {
   return (uint32_t)__cvta_generic_to_shared(p);
 }
-__device__ __forceinline__ uint64_t bsr_globaltimer() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
 __device__ __forceinline__ void bsr_mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
@@ -400,6 +419,7 @@ bsr_install_bulk_kernel(const __grid_constant__ BsrInstallParams p) {
   __shared__ int abort_flag;
 
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
+  bsr_span_begin(p.span_out, p.span_start);
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < BSR_K_BULK_STAGES; ++s) {

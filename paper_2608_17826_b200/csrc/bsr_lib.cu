@@ -77,6 +77,8 @@ struct JobRes {
   unsigned int *d_cnt = nullptr;  // [n_slots] CTA counters, kept zero
   unsigned int *h_err = nullptr;  // pinned, device-visible: raised by a kernel wait that gave up
   unsigned int *d_err = nullptr;  // device alias of h_err
+  uint64_t *d_span_start = nullptr;                  // [n_slots] scratch of the in-kernel span measurement, kept zero
+  uint64_t *h_span = nullptr, *d_span = nullptr;     // [n_slots] pinned, device-visible: span of the slot's last launch
   uint32_t n_slots = 0;
   uint64_t seq = 0;
 };
@@ -87,7 +89,7 @@ struct StatDelta {
            bytes_installed[BSR_MAX_RANKS] = {};
   uint64_t windows = 0, kernel_launches = 0, h2d_copies = 0, install_launches = 0,
            install_descriptors = 0;
-  double install_kernel_ms = 0.0;
+  double install_kernel_ms = 0.0, install_span_ms = 0.0;
 };
 
 // Host-side state of one restore through the slot pool.
@@ -243,6 +245,7 @@ void merge_stats(bsr_ctx *c, const StatDelta &d) {
   c->st.install_launches += d.install_launches;
   c->st.install_descriptors += d.install_descriptors;
   c->st.install_kernel_ms += d.install_kernel_ms;
+  c->st.install_span_ms += d.install_span_ms;
 }
 
 // ---- registration -> tile table (setup_mu held) --------------------------------------------------
@@ -371,6 +374,10 @@ void fill_params(bsr_ctx *c, BsrInstallParams &p, JobRes *res, uint32_t slot) {
   p.ctas_done = res->d_cnt + slot;
   p.err_flag = res->d_err;
   p.stall_tile = ~0u;
+  if (c->cfg.time_kernels) {
+    p.span_start = res->d_span_start + slot;
+    p.span_out = res->d_span + slot;
+  }
 }
 
 // host_source: the chunk is read from mapped host memory; plain loads are used for that.
@@ -428,6 +435,8 @@ void destroy_res(JobRes *res) {
   if (res->ev_done) cudaEventDestroy(res->ev_done);
   cudaFree(res->d_acc);
   cudaFree(res->d_cnt);
+  cudaFree(res->d_span_start);
+  if (res->h_span) cudaFreeHost(res->h_span);
   if (res->h_err) cudaFreeHost(res->h_err);
   if (res->stream) cudaStreamDestroy(res->stream);
 }
@@ -443,6 +452,11 @@ int init_scratch(bsr_ctx *c, JobRes *res, uint32_t n_slots) {
   CU(c, cudaHostAlloc((void **)&res->h_err, sizeof(unsigned int), cudaHostAllocMapped));
   CU(c, cudaHostGetDevicePointer((void **)&res->d_err, res->h_err, 0));
   *res->h_err = 0;
+  CU(c, cudaMalloc(&res->d_span_start, n_slots * 8));
+  CU(c, cudaMemset(res->d_span_start, 0, n_slots * 8));
+  CU(c, cudaHostAlloc((void **)&res->h_span, n_slots * 8, cudaHostAllocMapped));
+  CU(c, cudaHostGetDevicePointer((void **)&res->d_span, res->h_span, 0));
+  memset(res->h_span, 0, n_slots * 8);
   CU(c, cudaEventCreateWithFlags(&res->ev_done, cudaEventDisableTiming));
   std::lock_guard<std::mutex> g(c->mu);
   c->st.dev_aux_bytes += acc_bytes + cnt_bytes;
@@ -765,6 +779,7 @@ int restore_resident(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
   const uint32_t per_launch = BSR_K_MAX_BATCH / R ? BSR_K_MAX_BATCH / R : 1;
   int rc = BSR_OK;
   size_t n_timed = 0;
+  std::vector<uint32_t> span_slots;  // scratch sets of this call's launches (span measurement)
   // one descriptor per (chunk, rank) in launch order, uploaded once, ahead of the first launch
   for (uint32_t i = 0; i < N; ++i)
     for (uint32_t r = 0; r < R; ++r) {
@@ -784,7 +799,9 @@ int restore_resident(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
   for (uint32_t b0 = 0; b0 < N && rc == BSR_OK; b0 += per_launch) {
     const uint32_t b1 = (b0 + per_launch < N) ? b0 + per_launch : N;
     BsrInstallParams p{};
-    fill_params(c, p, res, R * c->cfg.dev_staging_depth + (uint32_t)(res->seq++ % kLaunchSlots));
+    const uint32_t slot = R * c->cfg.dev_staging_depth + (uint32_t)(res->seq++ % kLaunchSlots);
+    fill_params(c, p, res, slot);
+    if (c->cfg.time_kernels) span_slots.push_back(slot);
     p.n_adv = N;
     p.scatter = 1;
     p.tables = q->d_table_ptrs;
@@ -815,6 +832,9 @@ int restore_resident(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
     if (cudaEventElapsedTime(&ms, res->ev_pool[k].first, res->ev_pool[k].second) == cudaSuccess)
       sd.install_kernel_ms += ms;
   }
+  if (span_slots.size() <= kLaunchSlots)  // every launch had a scratch set of its own
+    for (size_t k = 0; k < span_slots.size(); ++k)
+      sd.install_span_ms += reinterpret_cast<volatile uint64_t *>(res->h_span)[span_slots[k]] * 1e-6;
   if (rc == BSR_OK) rc = wrc;
   if (rc != BSR_OK) return rc;
   for (uint32_t i = 0; i < N; ++i)
@@ -1019,6 +1039,7 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
         float ms = 0.f;
         if (cudaEventElapsedTime(&ms, res->ev_start[ls], res->ev_inst[ls]) == cudaSuccess)
           sd.install_kernel_ms += ms;
+        sd.install_span_ms += reinterpret_cast<volatile uint64_t *>(res->h_span)[ls] * 1e-6;
       }
       for (uint32_t s = L.first; s < L.first + L.count; ++s) {
         if (stages == kStagesAll) {
@@ -1755,6 +1776,8 @@ int bsr_restore_calibrate(bsr_ctx *c, bsr_req *q, int stages, double *seconds) {
   if (c->cfg.budget_slots == 0) serial.lock();
   *seconds = 0.0;
   if (q->n_adv == 0) return BSR_OK;
+  if (stages == BSR_CAL_FILL_H2D && c->cfg.direct_install)
+    return fail(c, BSR_ERR_STATE, "calibrate: a direct_install context has no device staging to copy into");
   CU(c, cudaSetDevice(c->cfg.device));
   JobRes *res = nullptr;
   int rc = acquire_res(c, &res);

@@ -91,8 +91,10 @@ def test_gpu_arm_prints_one_json_line_with_every_contract_key():
     assert r["launches"] == 3 * 2 and r["algorithmic_bytes_per_launch"] == 2 * 32 * 16_408_576
     assert abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9 and 0.2 < r["frac"] < 1.2
     assert abs(r["achieved"] - r["algorithmic_bytes_per_launch"] / r["avg_launch_ms"] / 1e6) < 1e-6
+    assert 0 < r["in_kernel"]["avg_span_ms"] < r["avg_launch_ms"]           # the kernel's own span lies inside the event pair
     res = d["resident"]
     assert res["descriptors_per_launch"] == 64 and 0.3 < res["frac"] < 1.2
+    assert 0 < res["in_kernel_span_ms"] < res["avg_launch_ms"]
     c = d["cpu_baseline"]
     assert c["kind"] == "oracle" and c["cores"] == 1 and c["value"] > 0 and c["sample"]
     assert c["all_cores"]["cores"] >= 1 and c["all_cores"]["value"] > 0

@@ -126,7 +126,9 @@ def test_restore_from_device_resident_tier(layout_name, R, N, W):
         gpu.request(keys, n_hit)
         assert gpu.restore() == gpu.B.BSR_OK, gpu.B.bsr_last_error(gpu.ctx)
         _check_success(case, W, gpu, ora, N)
-        assert gpu.stats().install_kernel_ms > 0
+        st = gpu.stats()
+        assert st.install_kernel_ms > 0
+        assert 0 < st.install_span_ms < st.install_kernel_ms      # the kernel's own span lies inside the event pair
 
 
 def test_library_computed_checksums_equal_oracle():
@@ -460,6 +462,10 @@ def test_calibration_passes_move_the_bytes_but_install_nothing():
                 for l in range(len(layout.tensors)):
                     assert bool((gpu.paged[r][l] == synth.CANARY).all())     # ... and no paged byte written
         assert B.bsr_restore_calibrate(gpu.ctx, gpu.req, 7)[0] == B.BSR_ERR_INVALID
+        with GpuSide(case, W, direct_install=True) as direct:           # no device staging to copy into
+            direct.request(keys, n_hit)
+            assert direct.B.bsr_restore_calibrate(direct.ctx, direct.req, B.BSR_CAL_FILL_H2D)[0] == B.BSR_ERR_STATE
+            assert direct.B.bsr_restore_calibrate(direct.ctx, direct.req, B.BSR_CAL_FILL)[0] == B.BSR_OK
         # a missing chunk fails a calibration pass like it fails a restore
         assert B.bsr_tier_remove(gpu.ctx, 1, keys[5]) == B.BSR_OK
         assert B.bsr_restore_calibrate(gpu.ctx, gpu.req, B.BSR_CAL_FILL)[0] == B.BSR_ERR_MISSING

@@ -35,7 +35,7 @@ def test_binding_covers_the_header_and_struct_sizes_match():
         assert callable(getattr(B, n))
     assert ctypes.sizeof(B.bsr_config) == 64  # as gcc lays out include/bsr.h
     assert ctypes.sizeof(B.bsr_tensor_desc) == 16
-    assert ctypes.sizeof(B.bsr_stats) == 8 * 8 * 5 + 8 * 7 + 8 * 4 + 8 * 2 + 8 * 2
+    assert ctypes.sizeof(B.bsr_stats) == 8 * 8 * 5 + 8 * 7 + 8 * 4 + 8 * 2 + 8 * 3
 
 
 def test_context_creation_fails_loudly_without_a_gpu_or_with_bad_arguments():
