@@ -586,6 +586,8 @@ def run_sweep(args):
 def spawn_ranks(args):
     """`python bench.py --gpus N` without a launcher: start one process per GPU (rank r drives GPU r),
     rendezvous on the loopback address, let rank 0's line through, return the worst exit code."""
+    from paper_2608_17826_b200 import build
+    build.build()  # once, before the ranks start
     with socket.socket() as s:
         s.bind(("127.0.0.1", 0))
         port = s.getsockname()[1]

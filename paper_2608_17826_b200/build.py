@@ -30,10 +30,16 @@ def up_to_date() -> bool:
 
 
 def _compile(out: str, defines: list[str], verbose: bool) -> str:
-    cmd = [nvcc(), *NVCC_FLAGS, *defines, "-o", out, SRC]
+    # built under a private name and renamed into place: several processes of one job (one per GPU)
+    # may find the library stale at the same moment, and none of them may load a half-written file
+    tmp = f"{out}.{os.getpid()}.tmp"
+    cmd = [nvcc(), *NVCC_FLAGS, *defines, "-o", tmp, SRC]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
+        if os.path.exists(tmp):
+            os.remove(tmp)
         raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
+    os.replace(tmp, out)
     if verbose:
         sys.stderr.write(res.stdout + res.stderr)
     return out

@@ -358,17 +358,20 @@ def test_install_kernel_in_use_reports_the_choice():
 
 # ---------------------------------------------------------------- many pipeline shapes
 def test_many_pipeline_shapes_give_the_same_bytes():
-    """Seeded sweep over W, fill threads, staging depth, install path and ranks on one small case:
-    ordering bugs in the slot pool / copy / install pipeline would show as a byte or bitmap mismatch."""
+    """Seeded sweep over W, fill threads, staging depth, chunks per install launch, install path and ranks
+    on two small registrations (long runs; long runs mixed with spans of short ones): ordering bugs in the
+    slot pool / copy / launch grouping / install pipeline would show as a byte or bitmap mismatch."""
     rng = np.random.default_rng(20260817)
-    layout = synth.Layout("mid", [64, 16], [(0, 1024), (0, 48), (1, 256)])
-    oracles = {}
-    for trial in range(16):
+    layouts = [synth.Layout("mid", [64, 16], [(0, 1024), (0, 48), (1, 256)]),
+               synth.Layout("mixed", [64, 16, 32], [(0, 512)] * 2 + [(1, 16)] * 40 + [(1, 64)] * 3 + [(2, 32)] * 9 + [(2, 272)])]
+    for trial in range(40):
+        layout = layouts[trial % 2]
         R = int(rng.integers(1, 4))
         N = int(rng.integers(1, 40))
-        W = int(rng.choice([1, 2, 3, 5, 8, 64]))
-        cfg = dict(load_concurrency=int(rng.choice([1, 2, 4, 8])), dev_staging_depth=int(rng.choice([1, 2, 4, 7])),
-                   install_variant=int(rng.choice([1, 2])), direct_install=bool(rng.integers(0, 2)))
+        W = int(rng.choice([1, 2, 3, 5, 8, 32, 64]))
+        cfg = dict(load_concurrency=int(rng.choice([1, 2, 4, 8])), dev_staging_depth=int(rng.choice([0, 1, 2, 4, 7])),
+                   install_variant=int(rng.choice([1, 2])), direct_install=bool(rng.integers(0, 3) == 0),
+                   install_batch=int(rng.choice([0, 1, 3, 8, 64])))
         case = Case(layout, R, N, seed=1400 + trial)
         ora = run_oracle(case, W)
         with GpuSide(case, W, **cfg) as gpu:
