@@ -321,7 +321,7 @@ typedef struct bsr_trace_rec {
   uint32_t chunk, rank, slot, reserved;
   uint64_t t_admit_ns;  /* a slot was reserved for the chunk (it becomes live)                  */
   uint64_t t_filled_ns; /* the last piece of the tier object landed in the slot                 */
-  uint64_t t_submit_ns; /* its copies and its install launch were queued                        */
+  uint64_t t_submit_ns; /* its copies were queued (its install launch follows when its group closes) */
   uint64_t t_done_ns;   /* its install was observed complete and the slot released; 0 = never   */
 } bsr_trace_rec;
 
