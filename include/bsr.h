@@ -329,6 +329,21 @@ typedef struct bsr_trace_rec {
  * admitted (chunk, rank), in admission order) into out[capacity]; *count = records available. */
 int bsr_get_trace(bsr_ctx *ctx, bsr_trace_rec *out, size_t capacity, size_t *count);
 
+/* How the install kernels cut one chunk of a registration into the spans they move (pure host code, no
+ * CUDA call; the same plan bsr_register's geometry gets at its first use).  A span is a contiguous
+ * byte range of the chunk of at most 16 KiB: either a piece of ONE destination run (n_runs == 1: bytes
+ * [dst_off, dst_off + bytes) of block `block` of tensor `tensor`), or n_runs whole runs of at most
+ * 1 KiB each that lie back to back in the chunk (run j is block (block + j) mod blocks-per-chunk of
+ * tensor `tensor` + (block + j) / blocks-per-chunk; all those tensors have the same bytes per token).
+ * dev_base of the tensor descriptors is ignored.  *count = spans of the plan; the first
+ * min(*count, capacity) are written to out.  Errors: INVALID, ALIGN as for bsr_register. */
+typedef struct bsr_span_info {
+  uint32_t src_off, bytes, dst_off, run_bytes;
+  uint32_t tensor, group, block, n_runs;
+} bsr_span_info;
+int bsr_plan_spans(const bsr_group_desc *groups, uint32_t n_groups, const bsr_tensor_desc *tensors,
+                   uint32_t n_tensors, bsr_span_info *out, size_t capacity, size_t *count);
+
 /* Host topology helper behind BSR_NUMA_AUTO (pure host code, no CUDA call): reads
  * <sysfs_root>/bus/pci/devices/<pci_bus_id>/numa_node into *node (-1 = the platform does not say),
  * counts the nodes under <sysfs_root>/devices/system/node into *n_nodes (may be NULL) and copies the

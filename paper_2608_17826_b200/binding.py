@@ -38,6 +38,7 @@ EXPORTS = [
     "bsr_probe_request", "bsr_req_bind", "bsr_request_done", "bsr_request_is_force_local",
     "bsr_get_trace", "bsr_tier_set_fetch", "bsr_restore_async", "bsr_restore_wait",
     "bsr_req_invalid_blocks", "bsr_install_kernel_in_use", "bsr_restore_calibrate", "bsr_numa_of_pci",
+    "bsr_plan_spans",
 ]
 # int fn(void *user, uint32 tier, uint32 rank, uint64 key, uint64 offset, uint64 len, void *dst)
 BSR_FETCH_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint64, C.c_uint64,
@@ -133,6 +134,8 @@ def _load() -> C.CDLL:
         "bsr_req_invalid_blocks": [vp, vp, u32, u32, vp, C.c_size_t, C.POINTER(C.c_size_t)],
         "bsr_install_kernel_in_use": [vp, C.POINTER(i32)],
         "bsr_restore_calibrate": [vp, vp, i32, C.POINTER(C.c_double)],
+        "bsr_plan_spans": [C.POINTER(bsr_group_desc), u32, C.POINTER(bsr_tensor_desc), u32, vp, C.c_size_t,
+                           C.POINTER(C.c_size_t)],
         "bsr_numa_of_pci": [C.c_char_p, C.c_char_p, C.POINTER(i32), C.c_char_p, C.c_size_t, C.POINTER(i32)],
     }
     for name, args in sig.items():
@@ -249,6 +252,18 @@ def bsr_restore_calibrate(ctx, req, stages: int):
     sec = C.c_double(0.0)
     rc = lib.bsr_restore_calibrate(ctx, req, stages, C.byref(sec))
     return rc, sec.value
+
+
+def bsr_plan_spans(block_tokens, tensors, capacity: int = 1 << 20):
+    """block_tokens: per group; tensors: [(group, bytes_per_token)].  Returns (rc, numpy structured array)
+    with one record per span of a chunk (host only, no CUDA call)."""
+    g = (bsr_group_desc * len(block_tokens))(*[bsr_group_desc(b, 1) for b in block_tokens])
+    t = (bsr_tensor_desc * len(tensors))(*[bsr_tensor_desc(gg, e, None) for gg, e in tensors])
+    dt = np.dtype([(k, "<u4") for k in ("src_off", "bytes", "dst_off", "run_bytes", "tensor", "group", "block", "n_runs")])
+    out = np.zeros(capacity, dtype=dt)
+    n = C.c_size_t(0)
+    rc = lib.bsr_plan_spans(g, len(block_tokens), t, len(tensors), out.ctypes.data, capacity, C.byref(n))
+    return rc, out[: min(n.value, capacity)]
 
 
 def bsr_numa_of_pci(sysfs_root: str, pci_bus_id: str):

@@ -279,9 +279,9 @@ bsr_install_vec_kernel(const __grid_constant__ BsrInstallParams p) {
 
 // ---------------------------------------------------------------------------------------------
 // install, bulk variant: the copy engine of each SM (1-D bulk async copies, one CTA each) moves the
-// tiles global -> shared -> global through a ring of shared-memory stages; a producer warp computes
-// addresses and issues the loads, a store warp issues the stores, and four warps sum the tile from
-// shared memory while its store is in flight.
+// spans global -> shared -> global through a ring of shared-memory stages; a producer warp computes
+// addresses and issues the loads, a store warp issues the stores, and the sum warps (4 or 8) sum the
+// span from shared memory while its store is in flight.
 //
 //   warp 0, producer:  wait empty[s] -> expect_tx(full[s], bytes) -> bulk load span into stage s
 //   warp 1, storer:    wait full[s]  -> bulk store stage s -> dst; once the store issued two spans

@@ -248,40 +248,44 @@ void merge_stats(bsr_ctx *c, const StatDelta &d) {
   c->st.install_span_ms += d.install_span_ms;
 }
 
-// ---- registration -> tile table (setup_mu held) --------------------------------------------------
-int finalize_registration(bsr_ctx *c) {
-  if (c->finalized.load(std::memory_order_acquire)) return BSR_OK;
-  if (c->L == 0) return fail(c, BSR_ERR_STATE, "no registration");
-  for (uint32_t r = 0; r < c->cfg.n_ranks; ++r)
-    if (!c->rank_registered[r]) return fail(c, BSR_ERR_STATE, "rank %u is not registered", r);
-  CU(c, cudaSetDevice(c->cfg.device));
-  std::vector<uint32_t> tgroup(c->L), trun(c->L);
+// ---- registration -> span table -----------------------------------------------------------------
+// Cuts one chunk into the spans the install kernels move (see BsrTile).  block_tokens per group;
+// group and bytes per token per tensor, group-major.
+void plan_spans(const std::vector<uint32_t> &block_tokens, const std::vector<uint32_t> &tensor_group,
+                const std::vector<uint32_t> &tensor_bpt, std::vector<BsrTile> &out) {
+  const uint32_t L = (uint32_t)tensor_group.size();
+  std::vector<uint64_t> seg_begin(block_tokens.size(), 0);
+  {
+    std::vector<bool> seen(block_tokens.size(), false);
+    uint64_t o = 0;
+    for (uint32_t l = 0; l < L; ++l) {
+      if (!seen[tensor_group[l]]) {
+        seen[tensor_group[l]] = true;
+        seg_begin[tensor_group[l]] = o;
+      }
+      o += (uint64_t)BSR_CHUNK_TOKENS * tensor_bpt[l];
+    }
+  }
   uint64_t off = 0;
-  c->h_tiles.clear();
-  for (uint32_t l = 0; l < c->L;) {
-    const TensorReg &t = c->tensors[l];
-    const uint32_t B = c->groups[t.group].block_tokens;
+  out.clear();
+  for (uint32_t l = 0; l < L;) {
+    const uint32_t group = tensor_group[l], bpt = tensor_bpt[l];
+    const uint32_t B = block_tokens[group];
     const uint32_t nb = BSR_CHUNK_TOKENS / B;
-    const uint64_t run = (uint64_t)B * t.bytes_per_token;
+    const uint64_t run = (uint64_t)B * bpt;
     const uint32_t run_inv = (uint32_t)(((1ull << 32) + run - 1) / run);
-    // a family: this tensor and the ones after it with the same group and bytes per token; their
-    // runs have one length and lie back to back in the chunk
     // Runs of up to BSR_K_SPAN_RUN_MAX bytes travel several to a span: below that a bulk copy per
     // run costs more in issue and stage turnover (about 150 ns per CTA) than its bytes are worth.
     const bool spans = run <= BSR_K_SPAN_RUN_MAX && 2 * run <= BSR_K_TILE_MAX;
+    // a family: this tensor and the ones after it with the same group and bytes per token; their
+    // runs have one length and lie back to back in the chunk
     uint32_t l_end = l + 1;
     if (spans)
-      while (l_end < c->L && c->tensors[l_end].group == t.group &&
-             c->tensors[l_end].bytes_per_token == t.bytes_per_token)
-        ++l_end;
-    for (uint32_t k = l; k < l_end; ++k) {
-      tgroup[k] = t.group;
-      trun[k] = (uint32_t)run;
-    }
+      while (l_end < L && tensor_group[l_end] == group && tensor_bpt[l_end] == bpt) ++l_end;
     BsrTile tl{};
     tl.run_bytes = (uint32_t)run;
     tl.run_inv = run_inv;
-    tl.group = (uint8_t)t.group;
+    tl.group = (uint8_t)group;
     if (spans) {
       // short runs: spans of as many whole runs as a stage holds, across the family's tensors
       const uint32_t per_span = (uint32_t)(BSR_K_TILE_MAX / run);
@@ -291,11 +295,11 @@ int finalize_registration(bsr_ctx *c) {
         tl.src_off = (uint32_t)(off + (uint64_t)v0 * run);
         tl.bytes = (uint32_t)(cnt * run);
         tl.dst_off = 0;
-        tl.word0 = (uint32_t)((tl.src_off - c->seg_begin[t.group]) / 4);
+        tl.word0 = (uint32_t)((tl.src_off - seg_begin[group]) / 4);
         tl.tensor = (uint16_t)(l + v0 / nb);
         tl.blk = (uint8_t)(v0 % nb);
         tl.n_runs = cnt;
-        c->h_tiles.push_back(tl);
+        out.push_back(tl);
       }
     } else {
       // long runs: each run on its own, cut into pieces of at most a stage
@@ -306,15 +310,38 @@ int finalize_registration(bsr_ctx *c) {
           tl.src_off = (uint32_t)(off + b * run + s);
           tl.bytes = (uint32_t)((run - s < piece) ? run - s : piece);
           tl.dst_off = (uint32_t)s;
-          tl.word0 = (uint32_t)((tl.src_off - c->seg_begin[t.group]) / 4);
+          tl.word0 = (uint32_t)((tl.src_off - seg_begin[group]) / 4);
           tl.tensor = (uint16_t)l;
           tl.blk = (uint8_t)b;
           tl.n_runs = 1;
-          c->h_tiles.push_back(tl);
+          out.push_back(tl);
         }
     }
-    off += (uint64_t)(l_end - l) * BSR_CHUNK_TOKENS * t.bytes_per_token;
+    off += (uint64_t)(l_end - l) * BSR_CHUNK_TOKENS * bpt;
     l = l_end;
+  }
+}
+
+// ---- registration -> tile table (setup_mu held) --------------------------------------------------
+int finalize_registration(bsr_ctx *c) {
+  if (c->finalized.load(std::memory_order_acquire)) return BSR_OK;
+  if (c->L == 0) return fail(c, BSR_ERR_STATE, "no registration");
+  for (uint32_t r = 0; r < c->cfg.n_ranks; ++r)
+    if (!c->rank_registered[r]) return fail(c, BSR_ERR_STATE, "rank %u is not registered", r);
+  CU(c, cudaSetDevice(c->cfg.device));
+  std::vector<uint32_t> tgroup(c->L), trun(c->L);
+  for (uint32_t l = 0; l < c->L; ++l) {
+    tgroup[l] = c->tensors[l].group;
+    trun[l] = c->groups[c->tensors[l].group].block_tokens * c->tensors[l].bytes_per_token;
+  }
+  {
+    std::vector<uint32_t> bt(c->G), tg(c->L), te(c->L);
+    for (uint32_t g = 0; g < c->G; ++g) bt[g] = c->groups[g].block_tokens;
+    for (uint32_t l = 0; l < c->L; ++l) {
+      tg[l] = c->tensors[l].group;
+      te[l] = c->tensors[l].bytes_per_token;
+    }
+    plan_spans(bt, tg, te, c->h_tiles);
   }
   // the kernels count the tiles of a launch (up to BSR_K_MAX_BATCH chunks) in 32 bits
   if (c->h_tiles.size() > (1u << 22))
@@ -1793,6 +1820,41 @@ int bsr_restore_calibrate(bsr_ctx *c, bsr_req *q, int stages, double *seconds) {
   *seconds = std::chrono::duration<double>(Clock::now() - t0).count();
   release_res(c, res);
   return rc;
+}
+
+int bsr_plan_spans(const bsr_group_desc *groups, uint32_t n_groups, const bsr_tensor_desc *tensors,
+                   uint32_t n_tensors, bsr_span_info *out, size_t capacity, size_t *count) {
+  if (!groups || !tensors || !count || (!out && capacity) || n_groups == 0 || n_groups > BSR_MAX_GROUPS ||
+      n_tensors == 0 || n_tensors > 65535)
+    return BSR_ERR_INVALID;
+  std::vector<uint32_t> bt(n_groups), tg(n_tensors), te(n_tensors);
+  for (uint32_t g = 0; g < n_groups; ++g) {
+    bt[g] = groups[g].block_tokens;
+    if (bt[g] == 0 || BSR_CHUNK_TOKENS % bt[g] || BSR_CHUNK_TOKENS / bt[g] > 255) return BSR_ERR_INVALID;
+  }
+  uint64_t per_token = 0;
+  for (uint32_t l = 0; l < n_tensors; ++l) {
+    tg[l] = tensors[l].group;
+    te[l] = tensors[l].bytes_per_token;
+    if (tg[l] >= n_groups || (l && tg[l] < tg[l - 1])) return BSR_ERR_INVALID;
+    if (te[l] == 0 || te[l] % 16) return BSR_ERR_ALIGN;
+    per_token += te[l];
+  }
+  if (per_token * BSR_CHUNK_TOKENS >= (1ull << 32)) return BSR_ERR_INVALID;
+  std::vector<BsrTile> tiles;
+  plan_spans(bt, tg, te, tiles);
+  *count = tiles.size();
+  for (size_t k = 0; k < tiles.size() && k < capacity; ++k) {
+    out[k].src_off = tiles[k].src_off;
+    out[k].bytes = tiles[k].bytes;
+    out[k].dst_off = tiles[k].dst_off;
+    out[k].run_bytes = tiles[k].run_bytes;
+    out[k].tensor = tiles[k].tensor;
+    out[k].group = tiles[k].group;
+    out[k].block = tiles[k].blk;
+    out[k].n_runs = tiles[k].n_runs;
+  }
+  return BSR_OK;
 }
 
 int bsr_numa_of_pci(const char *sysfs_root, const char *pci_bus_id, int *node, char *cpulist,
