@@ -928,7 +928,6 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
   };
   std::vector<Launch> launches;                // install launches issued, in order
   size_t launches_reaped = 0;                  // ... of which observed complete
-  std::vector<int64_t> buf_launch(R * D, -1);  // the launch that last read each staging buffer
   uint32_t live[BSR_MAX_RANKS] = {};
   uint64_t seen_done = 0;
   Inject inj;
@@ -1006,7 +1005,6 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
       first_error(fail(c, BSR_ERR_CUDA, "record: %s", cudaGetErrorString(e)));
       return;
     }
-    for (uint32_t s = first; s < first + n; ++s) buf_launch[(s % R) * D + (s / R) % D] = (int64_t)li;
     launches.push_back(Launch{first, n});
     launched = submitted;
   };
@@ -1084,7 +1082,7 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
     // submit, in order: every ready piece slot -> device staging on the copy stream; a chunk whose
     // pieces are all queued joins the open group, and a full group is launched
     while (!stop && submitted < admitted && submitted - reaped < R * D) {
-      const uint32_t i = submitted / R, r = submitted % R, d = i % D, k = r * D + d;
+      const uint32_t i = submitted / R, r = submitted % R, d = i % D;
       uint8_t *stage = direct ? nullptr : res->dstage[r] + (size_t)d * c->chunk_bytes;
       uint8_t *slot_host = c->ring[r] + (size_t)job.slot[submitted] * c->slot_bytes;
       cudaError_t e = cudaSuccess;
@@ -1104,11 +1102,9 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
         const uint64_t len = (c->chunk_bytes - off < kPieceBytes) ? c->chunk_bytes - off : kPieceBytes;
         const uint8_t *from = (o.loc == BSR_LOC_HOST) ? slot_host + off : o.data + off;
         if (!direct && stages != kStagesFill) {
-          // the staging buffer is free once the install launch that last read it has finished
-          if (cur_piece == 0 && stages == kStagesAll && buf_launch[k] >= (int64_t)launches_reaped)
-            e = cudaStreamWaitEvent(c->copy_stream, res->ev_inst[buf_launch[k] % n_ev], 0);
-          if (e == cudaSuccess)
-            e = cudaMemcpyAsync(stage + off, from, len, cudaMemcpyDefault, c->copy_stream);
+          // The staging buffer is free: its previous user, item submitted - R * D, lies in the reaped
+          // prefix (the loop condition above), so the launch that read it has been observed complete.
+          e = cudaMemcpyAsync(stage + off, from, len, cudaMemcpyDefault, c->copy_stream);
           if (e != cudaSuccess) {
             first_error(fail(c, BSR_ERR_TRANSFER, "copy submit: %s", cudaGetErrorString(e)));
             break;

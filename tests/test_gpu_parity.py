@@ -459,6 +459,7 @@ def test_calibration_passes_move_the_bytes_but_install_nothing():
             assert rc == B.BSR_OK and sec > 0
             st = gpu.stats()
             assert st.install_launches == 0 and st.bytes_installed[0] == 0
+            assert st.bytes_filled[0] == st.bytes_h2d[0] == st.h2d_copies == 0   # a calibration pass is not a restore
             assert st.peak_staging_bytes[0] == W * case.reg.slot_bytes       # the same slots were live
             assert gpu.commit() == 0 and (gpu.bitmap(N) == 0).all()          # nothing was installed ...
             for r in range(R):
