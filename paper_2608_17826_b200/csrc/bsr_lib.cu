@@ -1002,6 +1002,8 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
       }
     }
     if (e != cudaSuccess) {
+      // a launch without an event to observe it by: wait for it here, nothing may outlive the call
+      cudaStreamSynchronize(stream);
       first_error(fail(c, BSR_ERR_CUDA, "record: %s", cudaGetErrorString(e)));
       return;
     }
