@@ -9,18 +9,18 @@ launch shapes the benchmark times; configuration 3 once per window size, the ima
 on W).
 
 For configurations 4 and 5 (1,024-2,048 chunks, 16.8-33.6 GB per rank; and for the 1,024-chunk
-prefix of configuration 3 on a host with less than 100 GB free) the host tier holds P distinct seeded objects per rank
-and chunk i maps to object obj_of[i] (the first P chunks to objects 0..P-1, the rest drawn at
-random), so that the oracle can checksum every object.  The result is then checked through:
+prefix of configuration 3 on a host with less than 100 GB free) the host tier holds 71 distinct seeded
+objects per rank, so that the oracle can checksum every object, and the prefix is restored and checked
+TWICE: with chunk i pointing at object i mod 67, then at object i mod 71.  Each time:
   * every destination block of every tensor, gathered through the block table on the device,
     against the oracle's block of the object that chunk maps to;
   * every block outside the request's tables still holding the canary (the two together cover
     every byte of every pool);
   * every (rank, group, chunk) checksum the install kernel computed against the oracle's;
   * bitmap, exposure, windows, byte counters and the staging law.
-What this leaves to the materialised cases: a block written in the place of the same block of
-another chunk that maps to the same object cannot be told apart here.  The map is random, so a
-fault that misplaces chunks by any rule would have to hit such a pair every single time.
+A block written in the place of the same block of another chunk is invisible in one pass only if the
+two chunks point at the same object; 67 and 71 are coprime, so no two chunks of these prefixes do so in
+both passes.
 """
 import numpy as np
 import pytest
@@ -88,17 +88,19 @@ def test_short_run_registration_64_descriptors_per_launch_every_paged_byte():
 _OBJ_CACHE: dict = {}
 
 
+MAPS = (67, 71)   # chunk i -> object i mod 67 in the first pass, i mod 71 in the second
+
+
 class CyclicCase:
-    def __init__(self, layout, R, N, P, seed, present=None):
+    def __init__(self, layout, R, N, seed, present=None):
+        P = max(MAPS)
         self.layout, self.R, self.N, self.P, self.seed = layout, R, N, P, seed
         self.reg = O.Registration(list(layout.block_tokens), list(layout.tensors))
         self.G = self.reg.n_groups
         self.tok = synth.tokens(N * 256, seed=seed)
         self.salt = seed
         self.keys = O.prefix_keys(O.chunk_digests(self.tok, self.salt), self.salt, 1)
-        # chunk -> object: every object is used (the first P chunks), the rest is drawn at random
-        self.obj_of = np.concatenate([np.arange(min(P, N)),
-                                      np.random.default_rng(seed).integers(0, P, size=max(0, N - P))])
+        self.obj_of = np.arange(N) % MAPS[0]          # chunk -> object; use_map() switches to the second map
         ck = (layout.name, R, P)          # payload objects depend on the layout only: build them once
         if ck not in _OBJ_CACHE:
             objs = {(r, j): synth.chunk_payload(layout, r, j, seed=synth.MASTER_SEED + 1).copy()
@@ -128,13 +130,31 @@ class BigGpu:
             rc = B.bsr_register(self.ctx, r, [(case.layout.block_tokens[g], case.pools[g]) for g in range(case.G)],
                                 [(g, e, per[l].data_ptr()) for l, (g, e) in enumerate(case.layout.tensors)])
             assert rc == B.BSR_OK, B.bsr_last_error(self.ctx)
+        self.req = None
+        self.use_map(0)
+
+    def use_map(self, k):
+        """(Re)fills the tier: key of chunk i -> object i mod MAPS[k], with that object's stored checksums."""
+        B, case = self.B, self.case
+        case.obj_of = np.arange(case.N) % MAPS[k]
         for r in range(case.R):
             for i in range(case.N):
                 if case.present(r, i):
                     j = int(case.obj_of[i])
                     o = case.objs[(r, j)]
                     assert B.bsr_tier_put(self.ctx, r, case.keys[i], o, o.size, case.cks[(r, j)]) == B.BSR_OK
-        self.req = None
+
+    def restore_and_check_under_both_maps(self, W, n_adv):
+        """Restore and compare every block twice, the second time with every key pointing at another
+        object: 67 and 71 are coprime, so no two chunks of a prefix of up to 4,756 chunks share an
+        object in both passes, and a block written in another chunk's place shows in at least one."""
+        B = self.B
+        for k in range(len(MAPS)):
+            if k:
+                self.use_map(k)
+                B.bsr_reset_stats(self.ctx)
+            assert B.bsr_restore(self.ctx, self.req) == B.BSR_OK, B.bsr_last_error(self.ctx)
+            self.check_success(W, n_adv)
 
     def request(self, n_adv):
         c = self.case
@@ -267,7 +287,7 @@ def test_config3_materialised_every_paged_byte_for_each_window(N):
 def _config3_1024_chunks_with_the_object_map():
     N = 1024
     layout = synth.baseline_layout()
-    case = CyclicCase(layout, 2, N, P=67, seed=3003 + N)
+    case = CyclicCase(layout, 2, N, seed=3003 + N)
     g = read_golden("paper_capacity.txt")
     for W in (8, 16, 32, 64):
         gpu = BigGpu(case, W)
@@ -275,8 +295,7 @@ def _config3_1024_chunks_with_the_object_map():
             rc, keys, bm, n_hit = gpu.B.bsr_probe(gpu.ctx, case.tok, len(case.tok), case.salt)
             assert rc == gpu.B.BSR_OK and n_hit == N and np.array_equal(keys, case.keys)
             gpu.request(N)
-            assert gpu.B.bsr_restore(gpu.ctx, gpu.req) == gpu.B.BSR_OK, gpu.B.bsr_last_error(gpu.ctx)
-            gpu.check_success(W, N)
+            gpu.restore_and_check_under_both_maps(W, N)
             st = gpu.B.bsr_get_stats(gpu.ctx)[1]
             assert st.peak_staging_bytes[0] == st.peak_staging_bytes[1] == float(g[f"rws_mib_w{W}"]) * 2**20
         finally:
@@ -291,14 +310,13 @@ def test_config4_2048_chunks(layout_name):
     layout = {"baseline": synth.baseline_layout, "hetero": synth.hetero_layout,
               "mtp_on": synth.mtp_on_layout}[layout_name]()
     N, W = (2047 if layout_name == "mtp_on" else 2048), 32
-    case = CyclicCase(layout, 2, N, P=67, seed=4004)
+    case = CyclicCase(layout, 2, N, seed=4004)
     gpu = BigGpu(case, W)
     try:
         rc, keys, bm, n_hit = gpu.B.bsr_probe(gpu.ctx, case.tok, len(case.tok), case.salt)
         assert rc == gpu.B.BSR_OK and n_hit == N and np.array_equal(keys, case.keys)
         gpu.request(N)
-        assert gpu.B.bsr_restore(gpu.ctx, gpu.req) == gpu.B.BSR_OK, gpu.B.bsr_last_error(gpu.ctx)
-        gpu.check_success(W, N)
+        gpu.restore_and_check_under_both_maps(W, N)
         st = gpu.B.bsr_get_stats(gpu.ctx)[1]
         if layout_name == "mtp_on":
             assert st.peak_staging_bytes[0] == int(read_golden("paper_capacity.txt")["mtp_on_peak_w32"])
@@ -314,7 +332,7 @@ def test_config5_failures_at_1024_chunks(kind):
     layout = synth.baseline_layout()
     R, N, W = 2, 1024, 16
     present = (lambda r, i: i < 700 or i == 800) if kind == "partial_hit" else None
-    case = CyclicCase(layout, R, N, P=67, seed=5005, present=present)
+    case = CyclicCase(layout, R, N, seed=5005, present=present)
     gpu = BigGpu(case, W)
     B = gpu.B
     try:
@@ -324,8 +342,7 @@ def test_config5_failures_at_1024_chunks(kind):
             hit = np.array([i < 700 or i == 800 for i in range(N)])
             assert n_hit == 700 and np.array_equal(bm, O.pack_bits(hit))
             gpu.request(700)
-            assert B.bsr_restore(gpu.ctx, gpu.req) == B.BSR_OK
-            gpu.check_success(W, 700)
+            gpu.restore_and_check_under_both_maps(W, 700)
             st = B.bsr_get_stats(gpu.ctx)[1]
             assert st.windows == 44 and st.bytes_installed[0] == 11_486_003_200
             return
