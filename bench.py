@@ -527,6 +527,11 @@ def run_gpu(args):
         "resident": resident,
         "cpu_baseline": cpu,
         "clocks": clocks,
+        # the paper's own figures, on its hardware: context, not a target
+        "paper_context": {"hardware": "two DGX Spark nodes, TP = 2, Mooncake remote DRAM over 100 Gb/s RDMA / local SSD",
+                          "peak_staging_MiB_per_rank_at_W32": 500.75,
+                          "restore_ttft_s_512k_tokens_ssd_fs_concurrency_1_to_4": [43.1, 17.6],
+                          "restore_ttft_s_524k_tokens_remote_dram": 16.41},
     }
     print(json.dumps(out))
     if world > 1:
