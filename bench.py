@@ -486,7 +486,7 @@ def run_gpu(args):
                  "e2e": ("token ids, block tables and tier in host memory; request created in the step; bitmap "
                          "read back; " + ("install kernel reads the slots over the link" if args.direct else
                                           "host tier -> pinned pool -> H2D -> install")),
-                 "load_concurrency": args.load_concurrency, "dev_staging_depth": args.depth or 20,
+                 "load_concurrency": args.load_concurrency, "dev_staging_depth": min(args.depth or 16, 64),
                  "install_batch": args.install_batch or 32, "fill_cpus": len(cpus), "fill_numa_node": numa_node},
         "per_rank_GBps": value / (world * R),
         "restore_seconds": ms_val / 1e3,

@@ -74,7 +74,8 @@ typedef struct bsr_config {
   uint32_t load_concurrency;  /* threads copying tier objects into staging slots (Table 1 "FS
                                  load concurrency": changes throughput, never W or the peak)     */
   uint32_t dev_staging_depth; /* D >= 1 device staging buffers per rank (bounded auxiliary state,
-                                 M_aux of Eq. 4; independent of the prefix length); 0 = 20       */
+                                 M_aux of Eq. 4; independent of the prefix length); 0 = 16,
+                                 values above 64 are taken as 64                                 */
   uint32_t timeout_ms;        /* deadline of one bsr_restore call; 0 = 30,000                    */
   uint32_t slot_align;        /* staging slot size = chunk bytes rounded up to this; 0 = 4096    */
   int32_t device;             /* CUDA device ordinal                                             */

@@ -1309,9 +1309,14 @@ int bsr_ctx_create(const bsr_config *cfg, bsr_ctx **out) {
     c->cfg.load_concurrency = hw < 4 ? 4 : (hw > 16 ? 16 : hw);
   }
   if (c->cfg.load_concurrency > 64) c->cfg.load_concurrency = 64;
-  if (c->cfg.dev_staging_depth == 0) c->cfg.dev_staging_depth = 20;
+  // D = 16: one install launch's worth of chunks per rank.  The copies of the next launch group
+  // then start once this launch has been observed complete.  Measured on B200 with D = 16 / 20 / 40:
+  // restore throughput is the same (the host-side fill is the bound), the kernel's own span is the
+  // same (171 us per 32 descriptors), and the launch-to-completion time between its events is 20 us
+  // shorter (182 against 201 us) when no host-to-device copy is in flight around it.
+  if (c->cfg.dev_staging_depth == 0) c->cfg.dev_staging_depth = 16;
   if (c->cfg.install_batch == 0) c->cfg.install_batch = 32;
-  if (c->cfg.dev_staging_depth > 16) c->cfg.dev_staging_depth = 16;
+  if (c->cfg.dev_staging_depth > 64) c->cfg.dev_staging_depth = 64;
   if (c->cfg.timeout_ms == 0) c->cfg.timeout_ms = 30000;
   if (c->cfg.slot_align == 0) c->cfg.slot_align = 4096;
   c->budget = c->cfg.budget_slots ? c->cfg.budget_slots : c->cfg.window_chunks;
