@@ -54,13 +54,15 @@ LAYOUTS = {"baseline": synth.baseline_layout, "hetero": synth.hetero_layout, "mt
            "short_runs": synth.short_run_layout}
 
 
-def _config(n_chunks, layout_name="baseline"):
+def _config(n_chunks, layout_name="baseline", window=0):
     name = WORKLOAD["name"]
     if n_chunks != WORKLOAD["n_chunks"]:
         name = f"REDUCED to {n_chunks} chunks: " + name
     if layout_name != "baseline":
         name = f"LAYOUT {layout_name}: " + name
-    return {"workload": name, "rank_slices_per_gpu": WORKLOAD["n_ranks"], "W": WORKLOAD["W"],
+    if window and window != WORKLOAD["W"]:
+        name = f"WINDOW W={window} instead of {WORKLOAD['W']}: " + name
+    return {"workload": name, "rank_slices_per_gpu": WORKLOAD["n_ranks"], "W": window or WORKLOAD["W"],
             "l2": "every step moves 4.2 GB per GPU, far more than L2; no flush needed"}
 
 
@@ -351,7 +353,7 @@ def run_gpu(args):
             dist.init_process_group("nccl", device_id=dev)
 
     layout = LAYOUTS[args.layout]()
-    R, N, W = WORKLOAD["n_ranks"], args.chunks or WORKLOAD["n_chunks"], WORKLOAD["W"]
+    R, N, W = WORKLOAD["n_ranks"], args.chunks or WORKLOAD["n_chunks"], args.window or WORKLOAD["W"]
     chunk = layout.chunk_bytes
     # one request for the whole job: the same token ids everywhere; process p restores the rank
     # slices p, p + world, ... of the job's R * world slices
@@ -474,7 +476,7 @@ def run_gpu(args):
     else:
         cpu = {"value": None, "unit": UNIT, "cores": 0, "kind": "oracle", "sample": "timed at N = 1 only"}
 
-    cfg = _config(N, args.layout)
+    cfg = _config(N, args.layout, args.window)
     out = {
         **({"dry_run_one_gpu": True} if args.dry_run_one_gpu else {}),
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -486,8 +488,8 @@ def run_gpu(args):
                  "e2e": ("token ids, block tables and tier in host memory; request created in the step; bitmap "
                          "read back; " + ("install kernel reads the slots over the link" if args.direct else
                                           "host tier -> pinned pool -> H2D -> install")),
-                 "load_concurrency": args.load_concurrency, "dev_staging_depth": min(args.depth or 16, 64),
-                 "install_batch": args.install_batch or 32, "fill_cpus": len(cpus), "fill_numa_node": numa_node},
+                 "load_concurrency": args.load_concurrency, "dev_staging_depth": min(args.depth or max(2, (args.install_batch or 64) // R), 64),
+                 "install_batch": args.install_batch or 64, "fill_cpus": len(cpus), "fill_numa_node": numa_node},
         "per_rank_GBps": value / (world * R),
         "restore_seconds": ms_val / 1e3,
         "frac_of_h2d_link": value / world / h2d_gbs,
@@ -631,6 +633,7 @@ def main():
     ap.add_argument("--variant", type=int, default=0, help="install kernel: 0 auto, 1 vector, 2 bulk copy")
     ap.add_argument("--layout", default="baseline", choices=sorted(LAYOUTS),
                     help="registration geometry (the contract line is the baseline one)")
+    ap.add_argument("--window", type=int, default=0, help="window W in chunks (default: the workload's 32; the label says so)")
     ap.add_argument("--chunks", type=int, default=0, help="prefix length in chunks (default: the workload's 128)")
     ap.add_argument("--direct", action="store_true", help="staging-free install (kernel reads the pinned slots)")
     ap.add_argument("--dry-run-one-gpu", action="store_true",

@@ -74,8 +74,9 @@ typedef struct bsr_config {
   uint32_t load_concurrency;  /* threads copying tier objects into staging slots (Table 1 "FS
                                  load concurrency": changes throughput, never W or the peak)     */
   uint32_t dev_staging_depth; /* D >= 1 device staging buffers per rank (bounded auxiliary state,
-                                 M_aux of Eq. 4; independent of the prefix length); 0 = 16,
-                                 values above 64 are taken as 64                                 */
+                                 M_aux of Eq. 4; independent of the prefix length); 0 = what
+                                 one install launch takes per rank (install_batch / R, at least
+                                 2: 32 for the defaults at R = 2); values above 64 are taken as 64 */
   uint32_t timeout_ms;        /* deadline of one bsr_restore call; 0 = 30,000                    */
   uint32_t slot_align;        /* staging slot size = chunk bytes rounded up to this; 0 = 4096    */
   int32_t device;             /* CUDA device ordinal                                             */
@@ -95,12 +96,15 @@ typedef struct bsr_config {
                                  run concurrently and share a pool of B slots per rank; each holds
                                  at most W, together never more than B                            */
   uint32_t install_batch;     /* chunk descriptors (chunk x rank) one install launch takes on the
-                                 path through the slot pool; 0 = 32.  A launch waits until that many
-                                 chunks have been queued for copying: never more per rank than D or
-                                 W / 2, never fewer than one chunk of every rank, and never while
-                                 nothing else could make progress.  Larger launches run the kernel
-                                 nearer device-copy speed, smaller ones hand slots back sooner.
-                                 Changes throughput only, never W or the peak                      */
+                                 path through the slot pool; 0 = 64.  A launch waits until that many
+                                 chunks have been queued for copying: never more per rank than D,
+                                 never fewer than one chunk of every rank, and never while nothing
+                                 else could make progress.  It does not depend on W: a pinned slot
+                                 returns to the pool when its copy into device staging has been
+                                 observed complete, not when its launch has (with direct_install
+                                 the kernel reads the slots itself: one chunk per launch, slot held
+                                 until the launch is done).  Larger launches run the kernel nearer
+                                 device-copy speed.  Changes throughput only, never W or the peak */
   uint32_t numa_bind;         /* BSR_NUMA_*: placement of the fill threads and the pinned pool      */
 } bsr_config;
 
@@ -246,12 +250,15 @@ int bsr_req_release(bsr_ctx *ctx, bsr_req *req);
 
 /* Installs the advertised prefix of every rank.  Chunk i of rank r is copied from the tier into
  * a free pinned slot of r's pool (this restore holds at most W slots per rank; a slot is live from
- * its admission, before the fill, until its install has been observed complete), copied to a
- * device staging buffer on the library's copy stream, then verified and scattered through the
- * block tables by the install kernel on `cuda_stream` (a cudaStream_t, or NULL for a stream owned
- * by the library).  One install launch takes the chunks queued since the previous one (see
- * bsr_config.install_batch); their slots are released together when the launch has been observed
- * complete.  Objects that live in device memory are installed in place.  The first
+ * its admission, before the fill, until its copy into device staging has been observed complete:
+ * Eq. 3 bounds the pinned pool, the D staging buffers per rank are the bounded auxiliary state of
+ * Eq. 4), copied to a device staging buffer on the library's copy stream, then verified and
+ * scattered through the block tables by the install kernel on `cuda_stream` (a cudaStream_t, or
+ * NULL for a stream owned by the library).  One install launch takes the chunks queued since the
+ * previous one (see bsr_config.install_batch); a staging buffer is reused once the launch that read
+ * it has been observed complete.  With direct_install there is no device staging: the kernel reads
+ * the slot, which stays live until that launch is done.  Objects that live in device memory are
+ * installed in place.  The first
  * missing key, checksum mismatch, transfer error or deadline overrun stops admission, drains what
  * is in flight, invalidates the whole request and is returned.  Blocking; on return no slot is
  * live and every kernel of the call has finished.
@@ -323,7 +330,8 @@ typedef struct bsr_trace_rec {
   uint64_t t_admit_ns;  /* a slot was reserved for the chunk (it becomes live)                  */
   uint64_t t_filled_ns; /* the last piece of the tier object landed in the slot                 */
   uint64_t t_submit_ns; /* its copies were queued (its install launch follows when its group closes) */
-  uint64_t t_done_ns;   /* its install was observed complete and the slot released; 0 = never   */
+  uint64_t t_done_ns;   /* the slot went back to the pool: the chunk's copy into device staging (with
+                           direct_install: its install launch) was observed complete; 0 = never  */
 } bsr_trace_rec;
 
 /* Copies the timeline of the most recent restore that went through the slot pool (one record per

@@ -891,13 +891,13 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
   // Chunks of each rank that one install launch takes.  A launch costs about 13 us on top of its
   // bytes (read-only ramp, write-only tail, address look-ups, the last CTA's verdicts), so a single
   // 16 MB chunk (5 us of traffic) runs at a third of device-copy speed, 16 chunks at 0.72 and 32 at
-  // 0.88.  A launch never needs more staging buffers than a rank has, and leaves half of the window
-  // to the fill: measured on B200, restore throughput is the same with half the window waiting for
-  // its launch as with one chunk per launch (the fill threads only need a few free slots ahead),
-  // and the peak stays W slots either way.
+  // 0.88.  A launch never needs more staging buffers than a rank has.  A pinned slot goes back to the
+  // pool as soon as its copy into device staging has been observed complete, so the size of a launch
+  // does not depend on the window: W bounds the pinned slots (Eq. 3), D the device staging (M_aux).
+  // A kernel that reads the pinned slots itself (direct_install) holds them until it is done and
+  // takes one chunk per launch.
   uint32_t cpl = c->cfg.install_batch / R;
   if (cpl > D) cpl = D;
-  if (cpl > W / 2) cpl = W / 2;
   if (cpl > BSR_K_MAX_BATCH / R) cpl = BSR_K_MAX_BATCH / R;
   if (cpl == 0) cpl = 1;
   // items (chunk, rank) per launch; a kernel that reads pinned slots over the link takes one
@@ -922,7 +922,9 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
     c->jobs.push_back(&job);
   }
   // items are numbered s = i * R + r in admission order; each counter below is a prefix length
-  uint32_t admitted = 0, submitted = 0, launched = 0, reaped = 0, cur_piece = 0;
+  // admitted >= submitted >= launched >= reaped (install observed), submitted >= released (slot back
+  // in the pool) >= reaped
+  uint32_t admitted = 0, submitted = 0, launched = 0, reaped = 0, released = 0, cur_piece = 0;
   struct Launch {
     uint32_t first, count;
   };
@@ -951,6 +953,14 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
     c->free_slots[r].push_back(job.slot[s]);
     c->live_total[r]--;
   };
+  // Hands the slots of the items below `upto` back, in order (their bytes have left the slot).
+  auto release_upto = [&](uint32_t upto) {
+    for (; released < upto; ++released) {
+      job.trace[released].t_done_ns = now_ns();
+      release_slot(released);
+      live[released % R]--;
+    }
+  };
   // Closes the open group [launched, submitted): one install launch over all its descriptors.
   auto launch_group = [&]() {
     const uint32_t first = launched, n = submitted - launched;
@@ -962,10 +972,8 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
     } else if (stages == kStagesFillH2d) {
       e = cudaEventRecord(res->ev_inst[ls], c->copy_stream);
     } else {
-      if (!direct) {
-        e = cudaEventRecord(res->ev_h2d[ls], c->copy_stream);
-        if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, res->ev_h2d[ls], 0);
-      }
+      // the copy stream is in order: the copy event of the group's last item covers the whole group
+      if (!direct) e = cudaStreamWaitEvent(stream, res->ev_h2d[(first + n - 1) % (R * D)], 0);
       BsrInstallParams p{};
       fill_params(c, p, res, ls);
       p.n_adv = N;
@@ -1054,11 +1062,8 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
       if (e == cudaErrorNotReady) break;
       if (e != cudaSuccess) {
         first_error(fail(c, BSR_ERR_CUDA, "install event: %s", cudaGetErrorString(e)));
-        while (reaped < launched) {  // the context is unusable; nothing more can be observed
-          release_slot(reaped);
-          live[reaped % R]--;
-          ++reaped;
-        }
+        release_upto(submitted);  // the context is unusable; nothing more can be observed
+        reaped = launched;
         launches_reaped = launches.size();
         break;
       }
@@ -1068,18 +1073,33 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
           sd.install_kernel_ms += ms;
         sd.install_span_ms += reinterpret_cast<volatile uint64_t *>(res->h_span)[ls] * 1e-6;
       }
-      for (uint32_t s = L.first; s < L.first + L.count; ++s) {
-        if (stages == kStagesAll) {
+      if (stages == kStagesAll)
+        for (uint32_t s = L.first; s < L.first + L.count; ++s) {
           const int h = harvest(c, q, s % R, s / R, sd);
           if (h != BSR_OK) first_error(h);
         }
-        job.trace[s].t_done_ns = now_ns();
-        release_slot(s);
-        live[s % R]--;
-      }
+      release_upto(L.first + L.count);  // a finished launch has read its chunks, wherever they lay
       reaped = L.first + L.count;
       ++launches_reaped;
       progress = true;
+    }
+    // release, in order: a chunk whose copy into device staging has been observed complete no longer
+    // needs its pinned slot (the fill-only calibration queues no copy: the slot is free at once)
+    if (!direct) {
+      const uint32_t before = released;
+      while (released < submitted) {
+        if (stages != kStagesFill) {
+          const cudaError_t e = cudaEventQuery(res->ev_h2d[released % (R * D)]);
+          if (e == cudaErrorNotReady) break;
+          if (e != cudaSuccess) {
+            first_error(fail(c, BSR_ERR_CUDA, "copy event: %s", cudaGetErrorString(e)));
+            release_upto(submitted);
+            break;
+          }
+        }
+        release_upto(released + 1);
+      }
+      if (released != before) progress = true;
     }
     // submit, in order: every ready piece slot -> device staging on the copy stream; a chunk whose
     // pieces are all queued joins the open group, and a full group is launched
@@ -1120,6 +1140,15 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
         progress = true;
       }
       if (stop || blocked) break;
+      if (!direct && stages != kStagesFill) {
+        // Safe to record again: the event's previous item, submitted - R * D, lies in the reaped prefix.
+        e = cudaEventRecord(res->ev_h2d[submitted % (R * D)], c->copy_stream);
+        if (e != cudaSuccess) {
+          cudaStreamSynchronize(c->copy_stream);  // its copies are queued: nothing may outlive the call
+          first_error(fail(c, BSR_ERR_CUDA, "record: %s", cudaGetErrorString(e)));
+          break;
+        }
+      }
       const TierObj &o = job.objs[submitted];
       BsrChunkDesc &cd = q->h_desc[submitted];
       // direct mode: the kernel reads the pinned slot (or the device object) itself over the link
@@ -1149,19 +1178,23 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
         continue;
       }
       // A group that cannot grow must not wait to be full: every admitted chunk has been queued,
-      // nothing is in flight whose completion would free a slot, and admission is held up (the
-      // window is full, or other restores hold the rest of the pool).
+      // nothing is in flight whose completion would free a slot or a staging buffer, and admission
+      // is held up all the same (other restores hold the rest of the pool).
       if (!stop && submitted > launched && submitted == admitted && cur_piece == 0 &&
-          launches_reaped == launches.size()) {
+          released == submitted && launches_reaped == launches.size()) {
         launch_group();
         continue;
       }
-      // Sleep until a fill task of this restore finishes, or for a short while when there is an
-      // event to poll (the fill threads need the cores more than a spinning waiter does).
+      // Sleep until a fill task of this restore finishes, or for a short while when an event decides
+      // what happens next: an install launch in flight, or a copy whose slot the fill is waiting for
+      // (the fill threads need the cores more than a spinning waiter does).
       std::unique_lock<std::mutex> lk(c->fill_mu);
+      const bool fill_waits_for_a_slot = !stop && admitted < total && released < submitted &&
+                                         job.fill_next == job.fill_admitted;  // no piece left to hand out
       if (job.pieces_done == seen_done)
-        job.cv.wait_for(lk, launches_reaped < launches.size() ? std::chrono::microseconds(20)
-                                                              : std::chrono::microseconds(200));
+        job.cv.wait_for(lk, (launches_reaped < launches.size() || fill_waits_for_a_slot)
+                                ? std::chrono::microseconds(20)
+                                : std::chrono::microseconds(200));
       seen_done = job.pieces_done;
     }
   }
@@ -1181,8 +1214,8 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
       }
     c->rr = 0;
   }
-  // slots admitted but never installed go back to the pool
-  for (uint32_t s = reaped; s < admitted; ++s) release_slot(s);
+  // slots still held (their chunks never got as far as a finished copy or install) go back to the pool
+  for (uint32_t s = released; s < admitted; ++s) release_slot(s);
   {
     std::lock_guard<std::mutex> lk(c->mu);
     job.trace.resize(admitted);
@@ -1309,13 +1342,19 @@ int bsr_ctx_create(const bsr_config *cfg, bsr_ctx **out) {
     c->cfg.load_concurrency = hw < 4 ? 4 : (hw > 16 ? 16 : hw);
   }
   if (c->cfg.load_concurrency > 64) c->cfg.load_concurrency = 64;
-  // D = 16: one install launch's worth of chunks per rank.  The copies of the next launch group
-  // then start once this launch has been observed complete.  Measured on B200 with D = 16 / 20 / 40:
-  // restore throughput is the same (the host-side fill is the bound), the kernel's own span is the
-  // same (171 us per 32 descriptors), and the launch-to-completion time between its events is 20 us
-  // shorter (182 against 201 us) when no host-to-device copy is in flight around it.
-  if (c->cfg.dev_staging_depth == 0) c->cfg.dev_staging_depth = 16;
-  if (c->cfg.install_batch == 0) c->cfg.install_batch = 32;
+  // Defaults: 64 chunk descriptors per install launch and as many staging buffers as one launch
+  // group needs (D = 64 / R per rank: 32 at R = 2).  A group that uses every staging buffer makes the
+  // copies of the next group wait until its launch has been observed complete (0.35 ms per 19 ms
+  // of copying).  Measured on B200, restore from host memory, W = 32: throughput is the same with
+  // 32 / D = 16, 64 / D = 32 and 64 / D = 40 (48.6 / 48.5 / 48.5 GB/s: the host-side fill is the
+  // bound), the launches run at 0.88 / 0.95 / 0.90 of the HBM copy rate between their events and
+  // 0.94 / 0.98 / 0.98 by the kernel's own clock: a launch that meets a busy copy engine waits about
+  // 20 us longer for its start and its completion record.
+  if (c->cfg.install_batch == 0) c->cfg.install_batch = 64;
+  if (c->cfg.dev_staging_depth == 0) {
+    const uint32_t per_rank = c->cfg.install_batch / c->cfg.n_ranks;
+    c->cfg.dev_staging_depth = per_rank < 2 ? 2 : per_rank;
+  }
   if (c->cfg.dev_staging_depth > 64) c->cfg.dev_staging_depth = 64;
   if (c->cfg.timeout_ms == 0) c->cfg.timeout_ms = 30000;
   if (c->cfg.slot_align == 0) c->cfg.slot_align = 4096;

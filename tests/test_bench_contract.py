@@ -81,14 +81,14 @@ def test_gpu_arm_prints_one_json_line_with_every_contract_key():
     assert e["h2d_bytes_per_step"] >= payload + 32 * 256 * 4 and e["d2h_bytes_per_step"] > 0
     assert e["bound_GBps"] == min(e["h2d_link_GBps_measured"], e["host_fill_only_GBps"], e["host_fill_plus_h2d_GBps"])
     assert abs(e["frac_of_bound"] - e["value"] / e["bound_GBps"]) < 1e-9
-    # launches: one probe per step plus the install launches, 32 descriptors each on this workload
+    # launches: one probe per step plus the install launch (64 descriptors: all 32 chunks of both slices)
     inst = e["install"]
-    assert inst["descriptors_per_launch"] == 32 and inst["launches_per_step"] == 2
-    assert d["gpu_launches"] == 3 * (1 + 2)
+    assert inst["descriptors_per_launch"] == 64 and inst["launches_per_step"] == 1
+    assert d["gpu_launches"] == 3 * (1 + 1)
     assert set(("sm_mhz", "sm_max_mhz", "reasons")) <= set(d["clocks"])
     r = d["roofline"]
     assert r["bound"] == "hbm" and r["unit"] == "GB/s" and r["kernel"] == "bsr_install_bulk_kernel"
-    assert r["launches"] == 3 * 2 and r["algorithmic_bytes_per_launch"] == 2 * 32 * 16_408_576
+    assert r["launches"] == 3 and r["algorithmic_bytes_per_launch"] == 2 * 64 * 16_408_576
     assert abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9 and 0.2 < r["frac"] < 1.2
     assert abs(r["achieved"] - r["algorithmic_bytes_per_launch"] / r["avg_launch_ms"] / 1e6) < 1e-6
     assert 0 < r["in_kernel"]["avg_span_ms"] < r["avg_launch_ms"]           # the kernel's own span lies inside the event pair

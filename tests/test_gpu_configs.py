@@ -70,7 +70,7 @@ def test_short_run_registration_64_descriptors_per_launch_every_paged_byte():
     ora = run_oracle(case, W)
     assert ora["status"] == O.OK and ora["exposed"] == N
     for location, variant in ((0, 0), (1, 0), (1, 1)):
-        with GpuSide(case, W, location=location, install_variant=variant) as gpu:
+        with GpuSide(case, W, location=location, install_variant=variant, install_batch=32 if location == 0 else 0) as gpu:
             B = gpu.B
             rc, keys, bm, n_hit = gpu.probe()
             assert rc == B.BSR_OK and n_hit == N and np.array_equal(keys, ora["keys"])

@@ -386,11 +386,13 @@ def test_many_pipeline_shapes_give_the_same_bytes():
 
 # ---------------------------------------------------------------- install launches take several chunks
 @pytest.mark.parametrize("W,batch,depth,per_launch", [
-    (32, 0, 0, 32),     # defaults: 32 descriptors = 16 chunks of each of the 2 rank slices
-    (16, 0, 0, 16),     # ... but never more than half of the window per rank
+    (32, 0, 0, 64),     # defaults: 64 descriptors = 32 chunks of each of the 2 rank slices
+    (16, 0, 0, 64),     # ... whatever the window: a slot is free again once its copy has landed
+    (4, 0, 0, 64),
+    (1, 0, 0, 64),
     (16, 4, 0, 4),
     (16, 64, 3, 6),     # never more chunks per rank than staging buffers
-    (4, 0, 0, 4),
+    (2, 32, 16, 32),    # 16 chunks per rank per launch through a window of 2
     (16, 1, 0, 2),      # never less than one chunk of every rank slice
 ])
 def test_install_launches_carry_the_configured_number_of_chunks(W, batch, depth, per_launch):
@@ -647,10 +649,10 @@ def test_stores_of_long_runs_followed_by_a_long_stretch_of_short_run_spans_in_on
 
 
 def test_admission_stops_at_the_first_failure():
-    """After the failing chunk is observed nothing more is admitted: at most the chunks already in
-    the window were fetched, not the remaining hundreds."""
+    """After the failing chunk is observed nothing more is admitted: at most the chunks of its launch
+    group (up to D per rank) and those already in the window were fetched, not the remaining hundreds."""
     layout = synth.tiny_layout()
-    R, N, W, bad = 2, 300, 4, 6
+    R, N, W, bad, D = 2, 300, 4, 6, 32
     case = Case(layout, R, N, seed=1600)
     with GpuSide(case, W) as gpu:
         B = gpu.B
@@ -661,9 +663,9 @@ def test_admission_stops_at_the_first_failure():
         assert gpu.restore() == B.BSR_ERR_CHECKSUM
         st = gpu.stats()
         for r in range(R):
-            assert st.bytes_filled[r] <= (bad + 1 + 2 * W) * case.reg.chunk_bytes
-            assert st.bytes_h2d[r] <= (bad + 1 + 2 * W) * case.reg.chunk_bytes
-            assert st.bytes_installed[r] <= (bad + 1 + W) * case.reg.chunk_bytes
+            assert st.bytes_filled[r] <= (bad + 1 + D + 2 * W) * case.reg.chunk_bytes
+            assert st.bytes_h2d[r] <= (bad + 1 + D + 2 * W) * case.reg.chunk_bytes
+            assert st.bytes_installed[r] <= (bad + 1 + D) * case.reg.chunk_bytes
         assert gpu.commit() == 0 and (gpu.bitmap(N) == 0).all()
 
 

@@ -32,12 +32,12 @@ def test_install_kernel_reaches_its_stated_share_of_the_measured_copy_rate():
         assert out.returncode == 0, out.stderr[-2000:]
         d = json.loads([l for l in out.stdout.splitlines() if l.strip()][-1])
         # never a matter of timing: the launch shape and the staging law
-        assert d["roofline"]["descriptors_per_launch"] >= 32, d["roofline"]
+        assert d["roofline"]["descriptors_per_launch"] >= 64, d["roofline"]
         assert d["staging_residual_bytes"] == [0, 0]
         short = {}
         if d["resident"]["achieved"] < 0.70 * hbm:
             short["resident"] = d["resident"]["achieved"]
-        if d["roofline"]["achieved"] < 0.70 * hbm:  # 32 descriptors per launch: 0.88 of the copy rate measured
+        if d["roofline"]["achieved"] < 0.70 * hbm:  # 64 descriptors per launch: 0.95 of the copy rate measured
             short["in_restore"] = d["roofline"]["achieved"]
         if d["e2e"]["frac_of_h2d_link"] < 0.80:
             short["e2e"] = d["e2e"]["frac_of_h2d_link"]
