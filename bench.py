@@ -488,7 +488,7 @@ def run_gpu(args):
                  "e2e": ("token ids, block tables and tier in host memory; request created in the step; bitmap "
                          "read back; " + ("install kernel reads the slots over the link" if args.direct else
                                           "host tier -> pinned pool -> H2D -> install")),
-                 "load_concurrency": args.load_concurrency, "dev_staging_depth": min(args.depth or max(2, (args.install_batch or 64) // R), 64),
+                 "load_concurrency": args.load_concurrency, "dev_staging_depth": min(args.depth or max(16, (args.install_batch or 64) // R), 64),
                  "install_batch": args.install_batch or 64, "fill_cpus": len(cpus), "fill_numa_node": numa_node},
         "per_rank_GBps": value / (world * R),
         "restore_seconds": ms_val / 1e3,
@@ -511,7 +511,7 @@ def run_gpu(args):
         "staging_residual_bytes": [p - W * slot for p in peak_staging],
         "gpu_launches": int(st_val.kernel_launches),
         "roofline": {"bound": "hbm", "kernel": kernel_name,
-                     "what": "install launches inside the timed restore steps (a few chunks each, as they land)",
+                     "what": "install launches inside the timed restore steps (one per group of chunks whose copies have landed)",
                      "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
                      "frac": (achieved / hbm_peak) if achieved else None,
                      "traffic": traffic, "peak_source": peak_src,
@@ -555,8 +555,9 @@ def run_sweep(args):
     R, P, seed = 2, 67, synth.MASTER_SEED
     objs = {(r, j): synth.chunk_payload(layout, r, j, seed=seed).copy() for r in range(R) for j in range(P)}
     h2d = measure_h2d(torch, dev, layout.chunk_bytes)
-    plan = ([(N, W, 0, 0) for N in (512, 1024) for W in (8, 16, 32, 64)] + [(2048, 32, 0, 0)] +
-            [(512, 32, lc, 0) for lc in (1, 2, 4, 8, 16)] + [(512, W, 0, b) for W in (8, 32) for b in (2, 4, 8, 16)])
+    plan = ([(512, W, 0, 0) for W in (2, 4, 8, 16, 32, 64)] + [(1024, W, 0, 0) for W in (8, 16, 32, 64)] +
+            [(2048, 32, 0, 0)] + [(512, 32, lc, 0) for lc in (1, 2, 4, 8, 16)] +
+            [(512, 8, 0, b) for b in (2, 8, 32)])
     for N, W, lc, batch in plan:
         tok = synth.tokens(N * 256, seed=seed + N)
         payload = {(r, i): objs[(r, i % P)] for r in range(R) for i in range(N)}

@@ -76,7 +76,7 @@ typedef struct bsr_config {
   uint32_t dev_staging_depth; /* D >= 1 device staging buffers per rank (bounded auxiliary state,
                                  M_aux of Eq. 4; independent of the prefix length); 0 = what
                                  one install launch takes per rank (install_batch / R, at least
-                                 2: 32 for the defaults at R = 2); values above 64 are taken as 64 */
+                                 16: 32 for the defaults at R = 2); values above 64 are taken as 64 */
   uint32_t timeout_ms;        /* deadline of one bsr_restore call; 0 = 30,000                    */
   uint32_t slot_align;        /* staging slot size = chunk bytes rounded up to this; 0 = 4096    */
   int32_t device;             /* CUDA device ordinal                                             */
