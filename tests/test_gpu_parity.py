@@ -131,6 +131,39 @@ def test_restore_from_device_resident_tier(layout_name, R, N, W):
         assert 0 < st.install_span_ms < st.install_kernel_ms      # the kernel's own span lies inside the event pair
 
 
+@pytest.mark.parametrize("direct", [False, True])
+def test_tier_with_some_objects_in_device_memory_and_some_on_the_host(direct):
+    """A tier whose objects live partly in HBM and partly in host memory goes through the slot pool as a
+    whole: host objects are copied tier -> slot -> device, device objects device -> device (with
+    direct_install the kernel reads either in place); every paged byte as the oracle's, and only the
+    host objects count as filled."""
+    layout = synth.hetero_layout()
+    R, N, W = 2, 21, 4
+    case = Case(layout, R, N, seed=350)
+    ora = run_oracle(case, W)
+    with GpuSide(case, W, direct_install=direct) as gpu:
+        B, torch = gpu.B, gpu.torch
+        on_device = {(r, i): torch.from_numpy(case.payload[(r, i)]).to(gpu.dev)
+                     for r in range(R) for i in range(N) if (i + r) % 3 == 1}
+        for (r, i), t in on_device.items():     # the same key again: the index entry is replaced
+            assert B.bsr_tier_put(gpu.ctx, r, case.keys[i], t.data_ptr(), t.numel(), case.cks[(r, i)],
+                                  B.BSR_LOC_DEVICE) == B.BSR_OK
+        torch.cuda.synchronize()
+        rc, keys, bm, n_hit = gpu.probe()
+        assert rc == B.BSR_OK and n_hit == N
+        gpu.request(keys, n_hit)
+        assert gpu.restore() == B.BSR_OK, B.bsr_last_error(gpu.ctx)
+        assert gpu.commit() == ora["exposed"] == N
+        assert np.array_equal(gpu.bitmap(N), ora["req"].bitmap())
+        assert_paged_equal(gpu, ora["paged"])
+        st = gpu.stats()
+        for r in range(R):
+            n_host = sum(1 for i in range(N) if (r, i) not in on_device)
+            assert st.bytes_filled[r] == n_host * case.reg.chunk_bytes
+            assert st.bytes_installed[r] == N * case.reg.chunk_bytes
+            assert st.peak_staging_bytes[r] == W * case.reg.slot_bytes
+
+
 def test_library_computed_checksums_equal_oracle():
     for layout in (synth.tiny_layout(), synth.hetero_layout()):
         case = Case(layout, 2, 3, seed=400)
