@@ -399,7 +399,7 @@ int bsr_tier_remove_at(bsr_ctx *ctx, uint32_t tier, uint32_t rank, uint64_t key)
  * load_concurrency at once,
  *     fn(user, tier, rank, key, offset, len, dst)
  * to deliver bytes [offset, offset + len) of the object straight into the pinned staging slot at
- * dst (pieces of at most 8 MiB, in no particular order).  Return 0 on success; any other value
+ * dst (pieces of 1 to 8 MiB that tile the object, in no particular order).  Return 0 on success; any other value
  * fails the restore closed with BSR_ERR_TRANSFER.  fn must be thread-safe and must not call back
  * into the context.  NULL removes the adapter. */
 typedef int (*bsr_fetch_fn)(void *user, uint32_t tier, uint32_t rank, uint64_t key, uint64_t offset,

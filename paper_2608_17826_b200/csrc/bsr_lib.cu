@@ -17,6 +17,7 @@
 #include <sched.h>
 #include <sys/prctl.h>
 
+#include <algorithm>
 #include <atomic>
 #include <chrono>
 #include <condition_variable>
@@ -43,6 +44,14 @@ constexpr int kInstallThreads = 256;
 constexpr int kInstallUnroll = 2;  // 32 registers: 8 CTAs of 256 threads resident per SM
 constexpr int kLaunchSlots = 8;  // scratch sets for batched install launches in flight per restore
 constexpr uint64_t kPieceBytes = 8ull << 20;  // fill and host-to-device copy granularity
+// ... of the last chunks of a prefix.  When the fill threads finish their last pieces at about the same
+// time, everything they filled is still to be copied: with 8 threads and 8 MiB pieces up to 64 MiB,
+// more than a millisecond of link time after the last byte was fetched.  Small pieces, taken in order,
+// let the copies trail the fill closely where the restore ends.
+constexpr uint64_t kTailPieceBytes = 2ull << 20;
+// ... and of the first chunk of every rank: the copy engine has nothing to do until the first piece has
+// been fetched, and a short prefix is over before that millisecond has been made up for.
+constexpr uint64_t kHeadPieceBytes = 1ull << 20;
 #ifndef BSR_RING_ALLOC_FLAGS
 #define BSR_RING_ALLOC_FLAGS cudaHostAllocMapped
 #endif
@@ -92,11 +101,18 @@ struct StatDelta {
   double install_kernel_ms = 0.0, install_span_ms = 0.0;
 };
 
+// One fill task: a piece of one chunk of one rank, bytes [off, off + len) of the tier object.
+struct FillTask {
+  uint32_t item;  // chunk * R + rank
+  uint32_t off, len;
+};
+
 // Host-side state of one restore through the slot pool.
 struct Job {
   bsr_req *q = nullptr;
   Clock::time_point deadline;
-  uint32_t P = 1;
+  std::vector<FillTask> tasks;                // every piece of every item, in admission order
+  std::vector<uint32_t> task_begin;           // per (chunk, rank) item: index of its first piece; [n] = all pieces
   std::unique_ptr<std::atomic<int>[]> state;  // per piece: 0 pending, 1 ready, <0 error
   std::vector<TierObj> objs;                  // per (chunk, rank)
   std::vector<uint32_t> slot;                 // per (chunk, rank): slot of the rank's pool
@@ -160,7 +176,6 @@ struct bsr_ctx {
   std::vector<TensorReg> tensors;
   uint64_t chunk_bytes = 0, slot_bytes = 0;
   uint64_t seg_begin[BSR_MAX_GROUPS] = {}, seg_bytes[BSR_MAX_GROUPS] = {};
-  uint32_t pieces = 1;  // fill pieces per chunk
   std::atomic<bool> finalized{false};
   bool use_bulk = true;  // the install kernel chosen for this registration (see finalize_registration)
   bool has_spans = false;     // the tile table holds spans of several runs
@@ -595,11 +610,11 @@ void filler_main(bsr_ctx *c) {
       job->fill_active++;
     }
     bsr_req *req = job->q;
-    const uint32_t R = c->cfg.n_ranks, P = job->P;
-    const uint32_t s = t / P, piece = t % P;
+    const uint32_t R = c->cfg.n_ranks;
+    const FillTask ft = job->tasks[t];
+    const uint32_t s = ft.item, piece = t - job->task_begin[s];
     const uint32_t i = s / R, r = s % R;
-    const uint64_t off = (uint64_t)piece * kPieceBytes;
-    const uint64_t len = (c->chunk_bytes - off < kPieceBytes) ? c->chunk_bytes - off : kPieceBytes;
+    const uint64_t off = ft.off, len = ft.len;
     int state = 1;
     TierObj obj{};
     if (!job->abort.load(std::memory_order_acquire)) {
@@ -885,7 +900,6 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
   if (rc != BSR_OK) return rc;
   const uint32_t R = c->cfg.n_ranks, W = c->cfg.window_chunks, D = c->cfg.dev_staging_depth;
   const uint32_t N = q->n_adv, total = N * R;
-  const uint32_t P = c->pieces;
   const bool direct = c->cfg.direct_install != 0 && stages == kStagesAll;
   const uint32_t n_ev = res->n_slots;  // launch slots: a scratch set and three events each
   // Chunks of each rank that one install launch takes.  A launch costs about 13 us on top of its
@@ -906,12 +920,44 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
   Job job;
   job.q = q;
   job.deadline = deadline;
-  job.P = P;
-  job.state.reset(new std::atomic<int>[(size_t)total * P]);
-  for (size_t k = 0; k < (size_t)total * P; ++k) job.state[k].store(0, std::memory_order_relaxed);
+  // Pieces.  8 MiB in the body of a prefix.  1 MiB for the first chunk of every rank, so that the copy
+  // engine starts a fraction of a millisecond into the restore; from there the pieces grow by
+  // 512 KiB each, so that the fill threads, which all start at the same instant, finish theirs one
+  // after the other instead of in bursts of eight with the link idle in between.  2 MiB for the last
+  // items of the prefix, as many as the fill threads can have in the air at once.
+  {
+    const uint64_t in_air = (uint64_t)c->cfg.load_concurrency * kPieceBytes;
+    uint32_t n_tail = (uint32_t)((in_air + c->chunk_bytes - 1) / c->chunk_bytes);
+    n_tail = (n_tail + R - 1) / R * R;
+    if (n_tail > total) n_tail = total;
+    job.task_begin.resize((size_t)total + 1);
+    uint64_t ramp = kHeadPieceBytes;
+    for (uint32_t s = 0; s < total; ++s) {
+      job.task_begin[s] = (uint32_t)job.tasks.size();
+      for (uint64_t off = 0; off < c->chunk_bytes;) {
+        uint64_t want;
+        if (s < R) {
+          want = kHeadPieceBytes;
+        } else if (s + n_tail >= total) {
+          want = kTailPieceBytes;
+        } else {
+          if (ramp < kPieceBytes) ramp += 512u << 10;
+          want = ramp;
+        }
+        uint64_t len = c->chunk_bytes - off < want ? c->chunk_bytes - off : want;
+        if (c->chunk_bytes - off - len < (256u << 10)) len = c->chunk_bytes - off;  // no sliver at the end
+        job.tasks.push_back(FillTask{s, (uint32_t)off, (uint32_t)len});
+        off += len;
+      }
+    }
+    job.task_begin[total] = (uint32_t)job.tasks.size();
+  }
+  const size_t n_tasks = job.task_begin[total];
+  job.state.reset(new std::atomic<int>[n_tasks]);
+  for (size_t k = 0; k < n_tasks; ++k) job.state[k].store(0, std::memory_order_relaxed);
   job.objs.resize(total);
   job.slot.assign(total, 0);
-  job.t_piece.assign((size_t)total * P, 0);
+  job.t_piece.assign(n_tasks, 0);
   job.trace.assign(total, bsr_trace_rec{});
   job.t0 = Clock::now();
   auto now_ns = [&] {
@@ -1048,7 +1094,7 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
       if (n_new) {
         {
           std::lock_guard<std::mutex> lk(c->fill_mu);
-          job.fill_admitted = admitted * P;
+          job.fill_admitted = job.task_begin[admitted];
         }
         c->fill_cv.notify_all();
         progress = true;
@@ -1109,8 +1155,9 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
       uint8_t *slot_host = c->ring[r] + (size_t)job.slot[submitted] * c->slot_bytes;
       cudaError_t e = cudaSuccess;
       bool blocked = false;
+      const uint32_t t0 = job.task_begin[submitted], P = job.task_begin[submitted + 1] - t0;
       while (cur_piece < P) {
-        const int stt = job.state[(size_t)submitted * P + cur_piece].load(std::memory_order_acquire);
+        const int stt = job.state[(size_t)t0 + cur_piece].load(std::memory_order_acquire);
         if (stt == 0) {
           blocked = true;
           break;
@@ -1120,8 +1167,7 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
           break;
         }
         const TierObj &o = job.objs[submitted];
-        const uint64_t off = (uint64_t)cur_piece * kPieceBytes;
-        const uint64_t len = (c->chunk_bytes - off < kPieceBytes) ? c->chunk_bytes - off : kPieceBytes;
+        const uint64_t off = job.tasks[t0 + cur_piece].off, len = job.tasks[t0 + cur_piece].len;
         const uint8_t *from = (o.loc == BSR_LOC_HOST) ? slot_host + off : o.data + off;
         if (!direct && stages != kStagesFill) {
           // The staging buffer is free: its previous user, item submitted - R * D, lies in the reaped
@@ -1160,8 +1206,8 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
       cd.rank = r;
       for (uint32_t g = 0; g < BSR_MAX_GROUPS; ++g) cd.expect[g] = g < c->G ? o.ck[g] : 0;
       for (uint32_t pc = 0; pc < P; ++pc)
-        if (job.t_piece[(size_t)submitted * P + pc] > job.trace[submitted].t_filled_ns)
-          job.trace[submitted].t_filled_ns = job.t_piece[(size_t)submitted * P + pc];
+        if (job.t_piece[(size_t)t0 + pc] > job.trace[submitted].t_filled_ns)
+          job.trace[submitted].t_filled_ns = job.t_piece[(size_t)t0 + pc];
       job.trace[submitted].t_submit_ns = now_ns();
       ++submitted;
       cur_piece = 0;
@@ -1485,7 +1531,6 @@ int bsr_register(bsr_ctx *c, uint32_t rank, const bsr_group_desc *groups, uint32
       off += sz;
     }
     c->chunk_bytes = off;
-    c->pieces = (uint32_t)((off + kPieceBytes - 1) / kPieceBytes);
     c->slot_bytes = round_up(off, c->cfg.slot_align);
     c->st.slot_bytes = c->slot_bytes;
   } else {
