@@ -353,6 +353,23 @@ typedef struct bsr_span_info {
 int bsr_plan_spans(const bsr_group_desc *groups, uint32_t n_groups, const bsr_tensor_desc *tensors,
                    uint32_t n_tensors, bsr_span_info *out, size_t capacity, size_t *count);
 
+/* How a restore of n_chunks chunks of chunk_bytes bytes on n_ranks rank slices is cut into the pieces
+ * that its fill threads fetch (tier -> pinned slot, or the tier's fetch callback) and its copy stream
+ * moves, in the order they are handed out (pure host code, no CUDA call; the plan bsr_restore uses
+ * with fill_threads = load_concurrency).  Section 4 "Storage-side concurrency is orthogonal": the
+ * pieces change when bytes arrive, never how many slots are live.  The pieces of a chunk tile it in
+ * ascending offset order; 8 MiB in the body of a prefix, 1 MiB for the first chunk of every rank,
+ * growing by 512 KiB per piece from there, 2 MiB for the last chunks (as many as fill_threads pieces of
+ * 8 MiB cover), never under 256 KiB unless the chunk is.  *count = pieces of the plan; the first
+ * min(*count, capacity) are written to out.  Errors: INVALID (a zero argument, a chunk of 4 GiB or
+ * more, more than BSR_MAX_RANKS ranks, more than 2^24 items). */
+typedef struct bsr_piece_info {
+  uint32_t chunk, rank;   /* the chunk of the prefix and the rank slice the piece belongs to */
+  uint32_t offset, bytes; /* bytes [offset, offset + bytes) of that chunk                     */
+} bsr_piece_info;
+int bsr_plan_pieces(uint64_t chunk_bytes, uint32_t n_chunks, uint32_t n_ranks, uint32_t fill_threads,
+                    bsr_piece_info *out, size_t capacity, size_t *count);
+
 /* Host topology helper behind BSR_NUMA_AUTO (pure host code, no CUDA call): reads
  * <sysfs_root>/bus/pci/devices/<pci_bus_id>/numa_node into *node (-1 = the platform does not say),
  * counts the nodes under <sysfs_root>/devices/system/node into *n_nodes (may be NULL) and copies the

@@ -38,7 +38,7 @@ EXPORTS = [
     "bsr_probe_request", "bsr_req_bind", "bsr_request_done", "bsr_request_is_force_local",
     "bsr_get_trace", "bsr_tier_set_fetch", "bsr_restore_async", "bsr_restore_wait",
     "bsr_req_invalid_blocks", "bsr_install_kernel_in_use", "bsr_restore_calibrate", "bsr_numa_of_pci",
-    "bsr_plan_spans",
+    "bsr_plan_spans", "bsr_plan_pieces",
 ]
 # int fn(void *user, uint32 tier, uint32 rank, uint64 key, uint64 offset, uint64 len, void *dst)
 BSR_FETCH_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint64, C.c_uint64,
@@ -137,6 +137,7 @@ def _load() -> C.CDLL:
         "bsr_plan_spans": [C.POINTER(bsr_group_desc), u32, C.POINTER(bsr_tensor_desc), u32, vp, C.c_size_t,
                            C.POINTER(C.c_size_t)],
         "bsr_numa_of_pci": [C.c_char_p, C.c_char_p, C.POINTER(i32), C.c_char_p, C.c_size_t, C.POINTER(i32)],
+        "bsr_plan_pieces": [C.c_uint64, u32, u32, u32, vp, C.c_size_t, C.POINTER(C.c_size_t)],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -263,6 +264,16 @@ def bsr_plan_spans(block_tokens, tensors, capacity: int = 1 << 20):
     out = np.zeros(capacity, dtype=dt)
     n = C.c_size_t(0)
     rc = lib.bsr_plan_spans(g, len(block_tokens), t, len(tensors), out.ctypes.data, capacity, C.byref(n))
+    return rc, out[: min(n.value, capacity)]
+
+
+def bsr_plan_pieces(chunk_bytes: int, n_chunks: int, n_ranks: int, fill_threads: int, capacity: int = 1 << 20):
+    """Returns (rc, numpy structured array) with one record (chunk, rank, offset, bytes) per fill piece of a
+    restore, in the order the pieces are handed out (host only, no CUDA call)."""
+    dt = np.dtype([(k, "<u4") for k in ("chunk", "rank", "offset", "bytes")])
+    out = np.zeros(capacity, dtype=dt)
+    n = C.c_size_t(0)
+    rc = lib.bsr_plan_pieces(chunk_bytes, n_chunks, n_ranks, fill_threads, out.ctypes.data, capacity, C.byref(n))
     return rc, out[: min(n.value, capacity)]
 
 

@@ -814,6 +814,44 @@ int wait_event_deadline(bsr_ctx *c, cudaEvent_t ev, Clock::time_point deadline) 
   }
 }
 
+// ---- fill pieces ---------------------------------------------------------------------------------
+// Cuts the n_items (chunk, rank) items of a restore, in admission order (item = chunk * R + rank), into
+// the pieces the fill threads fetch and the copy stream moves.  8 MiB in the body of a prefix.  1 MiB
+// for the first chunk of every rank, so that the copy engine starts a fraction of a millisecond into
+// the restore; from there the pieces grow by 512 KiB each, so that the fill threads, which all start
+// at the same instant, finish theirs one after the other instead of in bursts with the link idle in
+// between.  2 MiB for the last items of the prefix, as many as the fill threads can have in the air
+// at once.  No piece is shorter than 256 KiB unless its chunk is.
+void plan_pieces(uint64_t chunk_bytes, uint32_t n_items, uint32_t R, uint32_t fill_threads,
+                 std::vector<FillTask> &tasks, std::vector<uint32_t> &task_begin) {
+  const uint64_t in_air = (uint64_t)fill_threads * kPieceBytes;
+  uint64_t n_tail = (in_air + chunk_bytes - 1) / chunk_bytes;
+  n_tail = (n_tail + R - 1) / R * R;
+  if (n_tail > n_items) n_tail = n_items;
+  tasks.clear();
+  task_begin.assign((size_t)n_items + 1, 0);
+  uint64_t ramp = kHeadPieceBytes;
+  for (uint32_t s = 0; s < n_items; ++s) {
+    task_begin[s] = (uint32_t)tasks.size();
+    for (uint64_t off = 0; off < chunk_bytes;) {
+      uint64_t want;
+      if (s < R) {
+        want = kHeadPieceBytes;
+      } else if (s + n_tail >= n_items) {
+        want = kTailPieceBytes;
+      } else {
+        if (ramp < kPieceBytes) ramp += 512u << 10;
+        want = ramp;
+      }
+      uint64_t len = chunk_bytes - off < want ? chunk_bytes - off : want;
+      if (chunk_bytes - off - len < (256u << 10)) len = chunk_bytes - off;  // no sliver at the end
+      tasks.push_back(FillTask{s, (uint32_t)off, (uint32_t)len});
+      off += len;
+    }
+  }
+  task_begin[n_items] = (uint32_t)tasks.size();
+}
+
 // ---- restore when every advertised chunk already lives in device memory --------------------------
 int restore_resident(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
                      Clock::time_point deadline, const std::vector<TierObj> &objs, StatDelta &sd) {
@@ -920,38 +958,7 @@ int restore_ring(bsr_ctx *c, bsr_req *q, JobRes *res, cudaStream_t stream,
   Job job;
   job.q = q;
   job.deadline = deadline;
-  // Pieces.  8 MiB in the body of a prefix.  1 MiB for the first chunk of every rank, so that the copy
-  // engine starts a fraction of a millisecond into the restore; from there the pieces grow by
-  // 512 KiB each, so that the fill threads, which all start at the same instant, finish theirs one
-  // after the other instead of in bursts of eight with the link idle in between.  2 MiB for the last
-  // items of the prefix, as many as the fill threads can have in the air at once.
-  {
-    const uint64_t in_air = (uint64_t)c->cfg.load_concurrency * kPieceBytes;
-    uint32_t n_tail = (uint32_t)((in_air + c->chunk_bytes - 1) / c->chunk_bytes);
-    n_tail = (n_tail + R - 1) / R * R;
-    if (n_tail > total) n_tail = total;
-    job.task_begin.resize((size_t)total + 1);
-    uint64_t ramp = kHeadPieceBytes;
-    for (uint32_t s = 0; s < total; ++s) {
-      job.task_begin[s] = (uint32_t)job.tasks.size();
-      for (uint64_t off = 0; off < c->chunk_bytes;) {
-        uint64_t want;
-        if (s < R) {
-          want = kHeadPieceBytes;
-        } else if (s + n_tail >= total) {
-          want = kTailPieceBytes;
-        } else {
-          if (ramp < kPieceBytes) ramp += 512u << 10;
-          want = ramp;
-        }
-        uint64_t len = c->chunk_bytes - off < want ? c->chunk_bytes - off : want;
-        if (c->chunk_bytes - off - len < (256u << 10)) len = c->chunk_bytes - off;  // no sliver at the end
-        job.tasks.push_back(FillTask{s, (uint32_t)off, (uint32_t)len});
-        off += len;
-      }
-    }
-    job.task_begin[total] = (uint32_t)job.tasks.size();
-  }
+  plan_pieces(c->chunk_bytes, total, R, c->cfg.load_concurrency, job.tasks, job.task_begin);
   const size_t n_tasks = job.task_begin[total];
   job.state.reset(new std::atomic<int>[n_tasks]);
   for (size_t k = 0; k < n_tasks; ++k) job.state[k].store(0, std::memory_order_relaxed);
@@ -1942,6 +1949,24 @@ int bsr_plan_spans(const bsr_group_desc *groups, uint32_t n_groups, const bsr_te
     out[k].group = tiles[k].group;
     out[k].block = tiles[k].blk;
     out[k].n_runs = tiles[k].n_runs;
+  }
+  return BSR_OK;
+}
+
+int bsr_plan_pieces(uint64_t chunk_bytes, uint32_t n_chunks, uint32_t n_ranks, uint32_t fill_threads,
+                    bsr_piece_info *out, size_t capacity, size_t *count) {
+  if (!count || (!out && capacity) || chunk_bytes == 0 || chunk_bytes >= (1ull << 32) || n_ranks == 0 ||
+      n_ranks > BSR_MAX_RANKS || fill_threads == 0 || (uint64_t)n_chunks * n_ranks > (1u << 24))
+    return BSR_ERR_INVALID;
+  std::vector<FillTask> tasks;
+  std::vector<uint32_t> begin;
+  plan_pieces(chunk_bytes, n_chunks * n_ranks, n_ranks, fill_threads, tasks, begin);
+  *count = tasks.size();
+  for (size_t k = 0; k < tasks.size() && k < capacity; ++k) {
+    out[k].chunk = tasks[k].item / n_ranks;
+    out[k].rank = tasks[k].item % n_ranks;
+    out[k].offset = tasks[k].off;
+    out[k].bytes = tasks[k].len;
   }
   return BSR_OK;
 }

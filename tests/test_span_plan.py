@@ -91,3 +91,50 @@ def test_span_counts_of_the_benchmarked_registrations():
     assert counts["baseline"] == (1292, 0)        # 56 x 4 runs in 5 pieces each + 43 x 4 runs of 2 KiB on their own
     assert counts["short_runs"] == (600, 400)     # 25,600 runs of 256 B, 64 to a span; 200 runs of 8 KiB
     assert counts["hetero"][1] > 0
+
+
+# ---------------------------------------------------------------- fill pieces of a restore
+MIB = 1 << 20
+
+
+@pytest.mark.parametrize("chunk,N,R,threads", [(16_408_576, 128, 2, 8), (16_408_576, 4, 2, 8), (16_408_576, 1, 1, 8),
+                                               (16_633_856, 37, 2, 3), (8_192_000, 32, 2, 16), (24_576, 300, 2, 8),
+                                               (327_680, 40, 8, 4), (100 * MIB + 16, 3, 1, 2)])
+def test_fill_pieces_tile_every_chunk_in_admission_order(chunk, N, R, threads):
+    """Host-only plan of the pieces a restore is fetched and copied in: every (chunk, rank) item tiled exactly,
+    items in admission order, piece sizes as the schedule states."""
+    from paper_2608_17826_b200 import binding as B
+    rc, p = B.bsr_plan_pieces(chunk, N, R, threads)
+    assert rc == B.BSR_OK and len(p) > 0
+    items = p["chunk"].astype(np.int64) * R + p["rank"]
+    assert (np.diff(items) >= 0).all() and sorted(set(items.tolist())) == list(range(N * R))   # admission order, none missing
+    for it in range(N * R):
+        q = p[items == it]
+        assert int(q["offset"][0]) == 0 and int(q["bytes"].sum()) == chunk                      # the chunk, exactly ...
+        assert (q["offset"][1:] == np.cumsum(q["bytes"].astype(np.int64))[:-1]).all()           # ... in ascending pieces
+    assert int(p["bytes"].max()) <= 8 * MIB
+    assert int(p["bytes"].min()) >= min(chunk, 256 << 10)                                       # no sliver
+    head = p[items < R]
+    assert int(head["bytes"].max()) <= MIB + (256 << 10)                                        # first chunk of every rank: 1 MiB
+    n_tail = min(N * R, -(-(-(-threads * 8 * MIB // chunk)) // R) * R)
+    tail = p[items >= N * R - n_tail]
+    assert int(tail["bytes"].max()) <= max(2 * MIB + (256 << 10), MIB + (256 << 10))            # last chunks: 2 MiB
+    body = p[(items >= R) & (items < N * R - n_tail)]
+    if len(body):
+        # from 1 MiB the wanted size grows by 512 KiB per piece up to 8 MiB and stays there; a piece is
+        # shorter only where its chunk ends
+        want = np.minimum(8 * MIB, MIB + (512 << 10) * (1 + np.arange(len(body), dtype=np.int64)))
+        ends_chunk = body["offset"].astype(np.int64) + body["bytes"] == chunk
+        assert (body["bytes"] <= want + (256 << 10)).all()
+        assert ((body["bytes"] == want) | ends_chunk).all()
+
+
+def test_fill_piece_plan_rejects_bad_arguments():
+    from paper_2608_17826_b200 import binding as B
+    assert B.bsr_plan_pieces(0, 4, 2, 8)[0] == B.BSR_ERR_INVALID
+    assert B.bsr_plan_pieces(1 << 32, 4, 2, 8)[0] == B.BSR_ERR_INVALID
+    assert B.bsr_plan_pieces(4096, 4, 0, 8)[0] == B.BSR_ERR_INVALID
+    assert B.bsr_plan_pieces(4096, 4, 9, 8)[0] == B.BSR_ERR_INVALID
+    assert B.bsr_plan_pieces(4096, 4, 2, 0)[0] == B.BSR_ERR_INVALID
+    rc, p = B.bsr_plan_pieces(4096, 0, 2, 8)
+    assert rc == B.BSR_OK and len(p) == 0
