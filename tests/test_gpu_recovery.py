@@ -238,6 +238,12 @@ def test_file_backed_lower_tier_through_the_fetch_adapter(tmp_path):
             pieces.sort()
             assert pieces[0][0] == 0 and sum(ln for _, ln in pieces) == layout.chunk_bytes
             assert all(a[0] + a[1] == b[0] for a, b in zip(pieces, pieces[1:]))
+        # ... and exactly the pieces the library's host-only plan lists for this restore
+        rc, plan = B.bsr_plan_pieces(layout.chunk_bytes, Nk, Rk, 4)
+        assert rc == B.BSR_OK
+        key_to_chunk = {int(k): i for i, k in enumerate(case.keys[:Nk])}
+        assert sorted((key_to_chunk[k], r, off, ln) for (_, r, k, off, ln) in calls) == \
+            sorted((int(q["chunk"]), int(q["rank"]), int(q["offset"]), int(q["bytes"])) for q in plan)
         # a read error on one rank: zero exposure, marker set
         fail_on[0] = (1, int(case.keys[3]))
         assert B.bsr_restore(ctx, req, None) == B.BSR_ERR_TRANSFER
