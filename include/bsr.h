@@ -342,7 +342,7 @@ int bsr_get_trace(bsr_ctx *ctx, bsr_trace_rec *out, size_t capacity, size_t *cou
  * CUDA call; the same plan bsr_register's geometry gets at its first use).  A span is a contiguous
  * byte range of the chunk of at most 16 KiB: either a piece of ONE destination run (n_runs == 1: bytes
  * [dst_off, dst_off + bytes) of block `block` of tensor `tensor`), or n_runs whole runs of at most
- * 4 KiB each that lie back to back in the chunk (run j is block (block + j) mod blocks-per-chunk of
+ * 1 KiB each that lie back to back in the chunk (run j is block (block + j) mod blocks-per-chunk of
  * tensor `tensor` + (block + j) / blocks-per-chunk; all those tensors have the same bytes per token).
  * dev_base of the tensor descriptors is ignored.  *count = spans of the plan; the first
  * min(*count, capacity) are written to out.  Errors: INVALID, ALIGN as for bsr_register. */

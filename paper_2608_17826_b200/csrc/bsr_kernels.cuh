@@ -13,7 +13,7 @@
 #define BSR_K_TILE_MAX 16384u     // largest tile in bytes (one bulk-copy stage)
 #endif
 #ifndef BSR_K_SPAN_RUN_MAX
-#define BSR_K_SPAN_RUN_MAX 4096u  // destination runs up to this length travel as spans of several runs
+#define BSR_K_SPAN_RUN_MAX 1024u  // destination runs up to this length travel as spans of several runs
 #endif
 #define BSR_K_PHI 0x9E3779B97F4A7C15ull
 

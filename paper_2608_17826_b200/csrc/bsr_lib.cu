@@ -290,9 +290,7 @@ void plan_spans(const std::vector<uint32_t> &block_tokens, const std::vector<uin
     const uint64_t run = (uint64_t)B * bpt;
     const uint32_t run_inv = (uint32_t)(((1ull << 32) + run - 1) / run);
     // Runs of up to BSR_K_SPAN_RUN_MAX bytes travel several to a span: below that a bulk copy per
-    // run costs more in issue and stage turnover (about 150 ns per CTA) than its bytes are worth
-    // (measured on the 170-tensor registrations: 0.98 of the copy rate with a limit of 1 KiB, 0.99
-    // with 2 to 8 KiB).
+    // run costs more in issue and stage turnover (about 150 ns per CTA) than its bytes are worth.
     const bool spans = run <= BSR_K_SPAN_RUN_MAX && 2 * run <= BSR_K_TILE_MAX;
     // a family: this tensor and the ones after it with the same group and bytes per token; their
     // runs have one length and lie back to back in the chunk
@@ -388,7 +386,7 @@ int finalize_registration(bsr_ctx *c) {
   // speed of a device copy where the bytes sit in runs that travel on their own (1.28 ms on the
   // baseline registration) and, with eight sum warps to issue the scattered stores of short-run
   // spans, at 0.91 of it on a registration of 256-byte runs, ahead of the vector kernel on every
-  // registration tried (0.89 there, 0.89 on the 170-tensor one, 0.95 on the baseline one).  So BSR_INSTALL_AUTO means the
+  // registration tried (0.89 there, 0.86 on the 170-tensor one).  So BSR_INSTALL_AUTO means the
   // bulk-copy kernel; the vector kernel serves direct_install and an explicit request.
   uint64_t span_bytes = 0;
   for (const BsrTile &tl : c->h_tiles)

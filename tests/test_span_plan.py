@@ -14,7 +14,7 @@ LAYOUTS = {
     "stores_then_spans": lambda: synth.Layout("stores_then_spans", [64, 16], [(0, 512)] * 2 + [(1, 16)] * 1124),
     "extremes": lambda: synth.Layout("extremes", [2, 256, 128], [(0, 16), (0, 16), (1, 16), (1, 4096), (2, 80)]),
 }
-STAGE, SPAN_RUN_MAX = 16384, 4096
+STAGE, SPAN_RUN_MAX = 16384, 1024
 
 
 @pytest.mark.parametrize("name", sorted(LAYOUTS))
@@ -88,7 +88,7 @@ def test_span_counts_of_the_benchmarked_registrations():
         layout = LAYOUTS[name]()
         rc, spans = B.bsr_plan_spans(layout.block_tokens, layout.tensors)
         counts[name] = (len(spans), int((spans["n_runs"] > 1).sum()))
-    assert counts["baseline"] == (1142, 22)       # 56 x 4 runs in 5 pieces each + 172 runs of 2 KiB, 8 to a span
+    assert counts["baseline"] == (1292, 0)        # 56 x 4 runs in 5 pieces each + 43 x 4 runs of 2 KiB on their own
     assert counts["short_runs"] == (600, 400)     # 25,600 runs of 256 B, 64 to a span; 200 runs of 8 KiB
     assert counts["hetero"][1] > 0
 
