@@ -79,7 +79,8 @@ struct Inject {
 struct JobRes {
   cudaStream_t stream = nullptr;                        // used when the caller passes no stream
   uint8_t *dstage[BSR_MAX_RANKS] = {};                  // D staging buffers per rank
-  std::vector<cudaEvent_t> ev_h2d, ev_inst, ev_start;   // [n_slots]: one set per install launch in flight
+  std::vector<cudaEvent_t> ev_h2d;                      // [n_slots >= R * D]: per staging buffer, the copy of its chunk
+  std::vector<cudaEvent_t> ev_inst, ev_start;           // [n_slots]: one pair per install launch in flight
   std::vector<std::pair<cudaEvent_t, cudaEvent_t>> ev_pool;  // launch timing, batched launches
   cudaEvent_t ev_done = nullptr;
   uint64_t *d_acc = nullptr;      // [n_slots][BATCH][GROUPS] checksum accumulators, kept zero
