@@ -427,6 +427,8 @@ def test_many_pipeline_shapes_give_the_same_bytes():
     (16, 64, 3, 6),     # never more chunks per rank than staging buffers
     (2, 32, 16, 32),    # 16 chunks per rank per launch through a window of 2
     (16, 1, 0, 2),      # never less than one chunk of every rank slice
+    (8, 256, 64, 96),   # the largest staging depth: the whole 48-chunk prefix of both slices in one launch
+    (8, 256, 200, 96),  # ... which is also what a larger request is taken as
 ])
 def test_install_launches_carry_the_configured_number_of_chunks(W, batch, depth, per_launch):
     layout = synth.Layout("mid", [64, 16], [(0, 1024), (0, 48), (1, 256)])
