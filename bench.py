@@ -436,6 +436,16 @@ def run_gpu(args):
         B.bsr_probe(side.ctx, tok, len(tok), salt, False)
     probe_us = (time.perf_counter() - t0) / 20 * 1e6
     numa_node = int(st_val.fill_numa_node)
+    # the failure path's scrub: zero-fill of every destination block of the request (the call blocks
+    # until the kernel has finished; the second call is the measured one)
+    scrub_ms = None
+    if side.req is not None:
+        for _ in range(2):
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            rc = B.bsr_invalidate(side.ctx, side.req, B.BSR_SCRUB)
+            scrub_ms = (time.perf_counter() - t0) * 1e3
+            assert rc == B.BSR_OK
     side.close()
 
     if rank != 0:
@@ -494,6 +504,10 @@ def run_gpu(args):
         "restore_seconds": ms_val / 1e3,
         "frac_of_h2d_link": value / world / h2d_gbs,
         "probe_host_us": probe_us,
+        "scrub": {"what": "bsr_invalidate(BSR_SCRUB) on the benchmarked request: host wall time of the call, "
+                          "zero-fill of all its destination blocks (write-only HBM traffic)",
+                  "ms": scrub_ms, "bytes": step_bytes,
+                  "write_GBps": step_bytes / (scrub_ms / 1e3) / 1e9 if scrub_ms else None},
         "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e, "host_wall_ms_per_step": wall_e2e,
                 "steps": e2e_steps,
                 "h2d_bytes_per_step": step_bytes + len(tok) * 4 + table_bytes,
