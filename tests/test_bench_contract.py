@@ -95,6 +95,7 @@ def test_gpu_arm_prints_one_json_line_with_every_contract_key():
     res = d["resident"]
     assert res["descriptors_per_launch"] == 64 and 0.3 < res["frac"] < 1.2
     assert 0 < res["in_kernel_span_ms"] < res["avg_launch_ms"]
+    assert d["scrub"]["bytes"] == payload and d["scrub"]["ms"] > 0          # the failure path's zero-fill, timed once
     c = d["cpu_baseline"]
     assert c["kind"] == "oracle" and c["cores"] == 1 and c["value"] > 0 and c["sample"]
     assert c["all_cores"]["cores"] >= 1 and c["all_cores"]["value"] > 0
